@@ -1,0 +1,13 @@
+"""CPU oracle (test infrastructure; never imported by the product path)."""
+from .indexer_topk import (  # noqa: F401
+    OracleResult,
+    decode,
+    decode_bf16,
+    decode_e4m3,
+    indexer_scores,
+    indexer_topk,
+    oracle_topk,
+    score_row,
+    select_topk,
+    visible_keys,
+)
