@@ -1,0 +1,155 @@
+/*
+ * lt_indexer.h -- C ABI of the fused DSA indexer top-k for NVIDIA B200 (sm_100a).
+ *
+ * The operation (paper Sec. 2, Eq. 1 and Sec. 3.1, Eq. 2): for every query row t
+ * of a prefill chunk and every key s it may see,
+ *
+ *     I[t, s] = k_scale[s] * sum_{j<H} w[t, j] * ReLU( q[t, j, :] . k[s, :] )
+ *
+ * and the result is, per row, the exact top-k keys by I, ordered by (score
+ * descending, key index ascending).  The T x N score matrix is never written
+ * to memory: a sample of the keys fixes equal-width score bins, candidates are
+ * gated against an online threshold bin while they are scored, only survivors
+ * are written back, and an exact select runs on the survivors (paper Sec. 3.2:
+ * sampling, filtering, threshold refresh, top-k selection).  Rows for which
+ * that scheme cannot guarantee exactness are recomputed by an unfused exact
+ * path, so the result is always the exact top-k of the library's own scores.
+ *
+ * Conventions for every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller; the library
+ *     never frees or keeps them.  Outputs are fully overwritten.
+ *   - Layouts are dense row-major: q[T][H][D], w[T][H] (fp32), k[N][D],
+ *     k_scale[N] (fp32), out_idx[T][topk] (int32), out_score[T][topk] (fp32).
+ *     q, k, w, k_scale must be 16-byte aligned.
+ *   - Row t stands at position causal_offset + t and sees keys
+ *     0 .. causal_offset + t inclusive, clipped to [0, N).  causal_offset >= N-1
+ *     disables masking.  Rows that see fewer than topk keys are padded with
+ *     index -1 and score -inf.
+ *   - Scores are computed from exact products of the stored values with fp32
+ *     accumulation; -0.0 is returned as +0.0.  Inputs must be finite (no NaN /
+ *     Inf, no e4m3 NaN codes) and k_scale >= 0; this is not checked.
+ *   - A query-side fp8 scale is folded by the caller into w (w[t,j] *= q_scale[t]),
+ *     which is exact because ReLU is positively homogeneous.
+ *   - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work on it
+ *     and never synchronise the host, except lt_read_status and the internal
+ *     arena growth of the 13-argument lt_indexer_topk.
+ *   - Return value: LT_OK or a negative LT_ERR_* code detected on the host
+ *     before anything is enqueued.  Conditions met on the device are recorded
+ *     in a status word (LT_STATUS_* bits) inside the workspace; kernels never
+ *     trap and every device-side wait is bounded.
+ */
+#ifndef LT_INDEXER_H_
+#define LT_INDEXER_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LT_VERSION 100
+
+/* storage type of q and k */
+#define LT_DTYPE_F32 0  /* float32                                   */
+#define LT_DTYPE_BF16 1 /* bfloat16 bit patterns                     */
+#define LT_DTYPE_E4M3 2 /* fp8 e4m3 ("fn") codes, k_scale required   */
+
+/* return codes */
+#define LT_OK 0
+#define LT_ERR_INVALID_ARG (-1) /* null pointer, size <= 0, topk > N or > LT_MAX_TOPK, misaligned pointer */
+#define LT_ERR_UNSUPPORTED (-2) /* dtype / shape the library has no path for                              */
+#define LT_ERR_WORKSPACE (-3)   /* workspace missing, misaligned or too small                             */
+#define LT_ERR_CUDA (-4)        /* a CUDA runtime call failed; see lt_last_cuda_error                     */
+
+/* bits of the device status word (lt_read_status, status[0]) */
+#define LT_STATUS_TIMEOUT 1  /* a bounded device-side wait ran out; results are invalid   */
+#define LT_STATUS_FALLBACK 2 /* some rows took the exact unfused fallback (informational) */
+#define LT_STATUS_BOUNDS 4   /* a debug bounds check failed                               */
+
+#define LT_MAX_TOPK 8192
+#define LT_BINS 256 /* m, the number of equal-width score bins (paper Sec. 3.2, "Sampling") */
+
+/* which implementation lt_indexer_topk_ex uses */
+#define LT_PATH_AUTO 0    /* fused tensor-core path when the shape allows it, else generic */
+#define LT_PATH_FUSED 1   /* fused tcgen05 path; LT_ERR_UNSUPPORTED if the shape does not fit */
+#define LT_PATH_GENERIC 2 /* generic SIMT scoring + full-row select (any H, D, dtype)      */
+
+/*
+ * Tunables.  None of them may change any output bit; they trade memory and speed.
+ * A zero field means "default".
+ */
+typedef struct lt_tunables {
+  int path;          /* LT_PATH_*                                                        */
+  int cap_mult;      /* candidate buffer capacity per row = cap_mult * topk (default 12,
+                        the paper's "conservative capacity 12k", Sec. 4.2)                */
+  int sample_mult;   /* sample size k' = sample_mult * topk (default 3, paper Sec. 3.2)  */
+  int segment_tiles; /* key tiles (128 keys each) per work item (default 256)            */
+  int grid;          /* CTAs of the scan kernel (default: number of SMs)                 */
+  int reserved[3];
+} lt_tunables;
+
+/*
+ * Fused indexer top-k (paper Sec. 3.2; Eq. 1 + Eq. 2), 13-argument form.
+ *   dtype is inferred: k_scale != NULL -> q, k are e4m3 codes; k_scale == NULL -> bf16.
+ *   out_score may be NULL.  Uses a library-owned workspace that grows on demand
+ *   (growth synchronises the device once); lt_shutdown frees it.
+ */
+int lt_indexer_topk(const void* q, const float* w, const void* k, const float* k_scale,
+                    int T, int N, int H, int D, int topk, int causal_offset,
+                    int32_t* out_idx, float* out_score, void* stream);
+
+/*
+ * General form: explicit dtype, caller-owned workspace (device memory, 256-byte
+ * aligned, at least lt_indexer_topk_workspace_bytes(...) bytes; its contents are
+ * scratch), optional tunables (NULL = defaults).  fp32 inputs are reachable only
+ * through this form.  The workspace also holds the status word.
+ */
+int lt_indexer_topk_ex(int dtype, const void* q, const float* w, const void* k, const float* k_scale,
+                       int T, int N, int H, int D, int topk, int causal_offset,
+                       int32_t* out_idx, float* out_score,
+                       void* workspace, size_t workspace_bytes, const lt_tunables* tunables, void* stream);
+
+/* Bytes of workspace lt_indexer_topk_ex needs for this problem (0 on invalid arguments). */
+size_t lt_indexer_topk_workspace_bytes(int dtype, int T, int N, int H, int D, int topk,
+                                       const lt_tunables* tunables);
+
+/*
+ * Dense scores of rows [row_begin, row_end) (Eq. 1), for debugging and parity:
+ * out_scores[(t - row_begin) * N + s] = I[t, s] for visible keys, -inf otherwise.
+ * The values are bit-identical to those lt_indexer_topk(_ex) ranks for the same
+ * dtype and path.  dtype as in lt_indexer_topk_ex; path = LT_PATH_*.
+ */
+int lt_indexer_scores(int dtype, const void* q, const float* w, const void* k, const float* k_scale,
+                      int T, int N, int H, int D, int causal_offset,
+                      int row_begin, int row_end, float* out_scores, int path, void* stream);
+
+/*
+ * Unfused baseline (the decoupled design of paper Sec. 1: materialise scores, then
+ * select): scores of `rows_per_pass` rows at a time are written to score_buf
+ * (device, >= rows_per_pass * N * 4 bytes), each pass followed by a full-row radix
+ * select.  Same outputs as lt_indexer_topk_ex.
+ */
+int lt_unfused_topk(int dtype, const void* q, const float* w, const void* k, const float* k_scale,
+                    int T, int N, int H, int D, int topk, int causal_offset,
+                    int32_t* out_idx, float* out_score,
+                    float* score_buf, size_t score_buf_bytes, int path, void* stream);
+
+/*
+ * Copies the 8-int status block of a workspace to host memory after synchronising
+ * `stream`: [0] LT_STATUS_* bits, [1] rows that took the fallback, [2] largest
+ * survivor count of any row, [3] total survivors (low 31 bits, saturating),
+ * [4] rows whose candidate buffer overflowed, [5..7] reserved.
+ * workspace == NULL reads the library-owned workspace of lt_indexer_topk.
+ */
+int lt_read_status(const void* workspace, int* status8_host, void* stream);
+
+const char* lt_strerror(int code);
+int lt_last_cuda_error(void); /* the cudaError_t behind the last LT_ERR_CUDA of this thread */
+int lt_version(void);
+void lt_shutdown(void); /* frees the library-owned workspace */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LT_INDEXER_H_ */

@@ -1,0 +1,180 @@
+"""ctypes binding of liblt_indexer.so: same names as the C ABI, argument marshalling only.
+
+Every function takes torch CUDA tensors (used purely as device memory), passes
+their pointers and sizes to the library and returns.  No arithmetic of the
+method happens here, and there is no fallback: if the library is missing the
+first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+LT_DTYPE_F32, LT_DTYPE_BF16, LT_DTYPE_E4M3 = 0, 1, 2
+LT_PATH_AUTO, LT_PATH_FUSED, LT_PATH_GENERIC = 0, 1, 2
+LT_OK = 0
+LT_STATUS_TIMEOUT, LT_STATUS_FALLBACK, LT_STATUS_BOUNDS = 1, 2, 4
+LT_MAX_TOPK = 8192
+
+_DTYPE_CODES = {"f32": LT_DTYPE_F32, "bf16": LT_DTYPE_BF16, "e4m3": LT_DTYPE_E4M3}
+
+
+class LtError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what} failed: {code} ({strerror(code)})")
+        self.code = code
+
+
+class Tunables(ctypes.Structure):
+    """Mirror of `lt_tunables`; zero fields mean "default"."""
+
+    _fields_ = [("path", ctypes.c_int), ("cap_mult", ctypes.c_int), ("sample_mult", ctypes.c_int),
+                ("segment_tiles", ctypes.c_int), ("grid", ctypes.c_int), ("reserved", ctypes.c_int * 3)]
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB_PATH
+
+
+def load() -> ctypes.CDLL:
+    """Loads the shared library (built in-tree by `build.build()`); raises if it is absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = library_path()
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: run `python -m paper_2607_11976_b200.build` (needs nvcc); "
+                           "there is no CPU or PyTorch fallback for this path")
+    lib = ctypes.CDLL(path)
+    vp, fp, ip, i, sz = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    lib.lt_indexer_topk.argtypes = [vp, fp, vp, fp, i, i, i, i, i, i, ip, fp, vp]
+    lib.lt_indexer_topk.restype = i
+    lib.lt_indexer_topk_ex.argtypes = [i, vp, fp, vp, fp, i, i, i, i, i, i, ip, fp, vp, sz, ctypes.POINTER(Tunables), vp]
+    lib.lt_indexer_topk_ex.restype = i
+    lib.lt_indexer_topk_workspace_bytes.argtypes = [i, i, i, i, i, i, ctypes.POINTER(Tunables)]
+    lib.lt_indexer_topk_workspace_bytes.restype = sz
+    lib.lt_indexer_scores.argtypes = [i, vp, fp, vp, fp, i, i, i, i, i, i, i, fp, i, vp]
+    lib.lt_indexer_scores.restype = i
+    lib.lt_unfused_topk.argtypes = [i, vp, fp, vp, fp, i, i, i, i, i, i, ip, fp, fp, sz, i, vp]
+    lib.lt_unfused_topk.restype = i
+    lib.lt_read_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int), vp]
+    lib.lt_read_status.restype = i
+    lib.lt_strerror.argtypes = [i]
+    lib.lt_strerror.restype = ctypes.c_char_p
+    lib.lt_last_cuda_error.restype = i
+    lib.lt_version.restype = i
+    lib.lt_shutdown.restype = None
+    _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load().lt_strerror(code).decode()
+
+
+def dtype_code(dtype) -> int:
+    return _DTYPE_CODES[dtype] if isinstance(dtype, str) else int(dtype)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(code: int, what: str) -> None:
+    if code != LT_OK:
+        extra = f" (cudaError {load().lt_last_cuda_error()})" if code == -4 else ""
+        raise LtError(code, what + extra)
+
+
+def _shape(q: torch.Tensor, k: torch.Tensor):
+    T, H, D = q.shape
+    N, D2 = k.shape
+    if D2 != D:
+        raise ValueError("q and k disagree on D")
+    return T, N, H, D
+
+
+def lt_indexer_topk_workspace_bytes(dtype, T: int, N: int, H: int, D: int, topk: int,
+                                    tunables: Optional[Tunables] = None) -> int:
+    return int(load().lt_indexer_topk_workspace_bytes(dtype_code(dtype), T, N, H, D, topk,
+                                                      ctypes.byref(tunables) if tunables else None))
+
+
+def lt_indexer_topk(q, w, k, k_scale, topk: int, causal_offset: int, out_idx, out_score=None, stream=None) -> None:
+    """13-argument C entry point: dtype inferred from k_scale (None -> bf16, else e4m3)."""
+    T, N, H, D = _shape(q, k)
+    _check(load().lt_indexer_topk(_ptr(q), _ptr(w), _ptr(k), _ptr(k_scale), T, N, H, D, topk, causal_offset,
+                                  _ptr(out_idx), _ptr(out_score), _stream(stream)), "lt_indexer_topk")
+
+
+def lt_indexer_topk_ex(dtype, q, w, k, k_scale, topk: int, causal_offset: int, out_idx, out_score, workspace,
+                       tunables: Optional[Tunables] = None, stream=None) -> None:
+    T, N, H, D = _shape(q, k)
+    _check(load().lt_indexer_topk_ex(dtype_code(dtype), _ptr(q), _ptr(w), _ptr(k), _ptr(k_scale), T, N, H, D, topk,
+                                     causal_offset, _ptr(out_idx), _ptr(out_score), _ptr(workspace),
+                                     workspace.numel() * workspace.element_size(),
+                                     ctypes.byref(tunables) if tunables else None, _stream(stream)), "lt_indexer_topk_ex")
+
+
+def lt_indexer_scores(dtype, q, w, k, k_scale, causal_offset: int, row_begin: int, row_end: int, out_scores,
+                      path: int = LT_PATH_AUTO, stream=None) -> None:
+    T, N, H, D = _shape(q, k)
+    _check(load().lt_indexer_scores(dtype_code(dtype), _ptr(q), _ptr(w), _ptr(k), _ptr(k_scale), T, N, H, D, causal_offset,
+                                    row_begin, row_end, _ptr(out_scores), path, _stream(stream)), "lt_indexer_scores")
+
+
+def lt_unfused_topk(dtype, q, w, k, k_scale, topk: int, causal_offset: int, out_idx, out_score, score_buf,
+                    path: int = LT_PATH_AUTO, stream=None) -> None:
+    T, N, H, D = _shape(q, k)
+    _check(load().lt_unfused_topk(dtype_code(dtype), _ptr(q), _ptr(w), _ptr(k), _ptr(k_scale), T, N, H, D, topk,
+                                  causal_offset, _ptr(out_idx), _ptr(out_score), _ptr(score_buf),
+                                  score_buf.numel() * score_buf.element_size(), path, _stream(stream)), "lt_unfused_topk")
+
+
+def lt_read_status(workspace=None, stream=None) -> list:
+    """Synchronises the stream and returns the 8-int status block of a workspace
+    (None: the library-owned workspace of lt_indexer_topk)."""
+    buf = (ctypes.c_int * 8)()
+    _check(load().lt_read_status(_ptr(workspace), buf, _stream(stream)), "lt_read_status")
+    return list(buf)
+
+
+# ---------------------------------------------------------------------------------------------
+# device-memory helpers (plumbing only)
+# ---------------------------------------------------------------------------------------------
+
+def to_device(inp, device="cuda"):
+    """Uploads a workload (numpy storage codes) as torch tensors: (q, w, k, k_scale)."""
+    def up(a):
+        return None if a is None else torch.from_numpy(a).to(device)
+
+    if inp.dtype == "bf16":
+        q = torch.from_numpy(inp.q.view("int16")).to(device).view(torch.bfloat16)
+        k = torch.from_numpy(inp.k.view("int16")).to(device).view(torch.bfloat16)
+    else:
+        q, k = up(inp.q), up(inp.k)
+    return q, up(inp.w), k, up(inp.k_scale)
+
+
+def alloc_workspace(dtype, T, N, H, D, topk, tunables: Optional[Tunables] = None, device="cuda") -> torch.Tensor:
+    nbytes = lt_indexer_topk_workspace_bytes(dtype, T, N, H, D, topk, tunables)
+    if nbytes == 0:
+        raise ValueError("invalid problem for lt_indexer_topk_workspace_bytes")
+    return torch.empty(nbytes, dtype=torch.uint8, device=device)

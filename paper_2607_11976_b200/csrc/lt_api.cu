@@ -1,0 +1,502 @@
+// C ABI of the indexer top-k library: argument checks, workspace layout, kernel sequencing.
+#include <cuda_runtime.h>
+#include <limits.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <mutex>
+
+#include "../../include/lt_indexer.h"
+#include "lt_common.cuh"
+#include "lt_host.h"
+
+namespace lt {
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+
+#define LT_CUDA(expr)                                  \
+  do {                                                 \
+    cudaError_t e__ = (expr);                          \
+    if (e__ != cudaSuccess) {                          \
+      g_last_cuda_error = static_cast<int>(e__);       \
+      return LT_ERR_CUDA;                              \
+    }                                                  \
+  } while (0)
+
+constexpr size_t kAlign = 256;
+size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+
+constexpr size_t kFallbackScratchBudget = size_t(512) << 20;  // dense scores kept at once by the exact fallback
+constexpr size_t kGenericScratchBudget = size_t(256) << 20;   // dense scores kept at once by the generic path
+
+struct Tun {
+  int path, cap_mult, sample_mult, segment_tiles, grid;
+};
+Tun resolve_tunables(const lt_tunables* t) {
+  Tun r{LT_PATH_AUTO, 12, 3, 0, 0};
+  if (t != nullptr) {
+    r.path = t->path;
+    if (t->cap_mult > 0) r.cap_mult = t->cap_mult;
+    if (t->sample_mult > 0) r.sample_mult = t->sample_mult;
+    if (t->segment_tiles > 0) r.segment_tiles = t->segment_tiles;
+    if (t->grid > 0) r.grid = t->grid;
+  }
+  return r;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_problem(int dtype, const void* q, const float* w, const void* k, const float* k_scale, int T, int N, int H, int D) {
+  if (dtype != LT_DTYPE_F32 && dtype != LT_DTYPE_BF16 && dtype != LT_DTYPE_E4M3) return LT_ERR_UNSUPPORTED;
+  if (q == nullptr || w == nullptr || k == nullptr) return LT_ERR_INVALID_ARG;
+  if (dtype == LT_DTYPE_E4M3 && k_scale == nullptr) return LT_ERR_INVALID_ARG;
+  if (T <= 0 || N <= 0 || H <= 0 || D <= 0) return LT_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(w) || !aligned16(k) || (k_scale != nullptr && !aligned16(k_scale))) return LT_ERR_INVALID_ARG;
+  if (static_cast<size_t>(H) * D * 4 + 128 * (static_cast<size_t>(D) + 1) * 4 > 200 * 1024) return LT_ERR_UNSUPPORTED;
+  return LT_OK;
+}
+
+bool use_fused(const Tun& tun, int dtype, int H, int D) {
+  return tun.path != LT_PATH_GENERIC && scan_mma_supported(dtype, H, D);
+}
+
+// ---- workspace layout ------------------------------------------------------------------------
+struct Layout {
+  bool fused;
+  // zeroed region
+  size_t ctl, tail, hist, row_flag, block_flag, zero_end;
+  size_t smin, width, thr, fb_list, sample, cand, scratch, total;
+  int cap, n_sample, sample_stride, fb_slots, n_blocks, generic_rows;
+};
+
+Layout make_layout(bool fused, int T, int N, int topk, int causal_offset, const Tun& tun) {
+  Layout L{};
+  L.fused = fused;
+  size_t off = 0;
+  L.ctl = off;
+  off = align_up(off + sizeof(Control));
+  if (!fused) {
+    long long rows = static_cast<long long>(kGenericScratchBudget / (static_cast<size_t>(N) * 4));
+    L.generic_rows = static_cast<int>(rows < 1 ? 1 : (rows > T ? T : rows));
+    L.zero_end = off;
+    L.scratch = off;
+    off = align_up(off + static_cast<size_t>(L.generic_rows) * N * 4);
+    L.total = off;
+    return L;
+  }
+  L.n_blocks = (T + kRowsPerBlock - 1) / kRowsPerBlock;
+  L.tail = off;
+  off = align_up(off + static_cast<size_t>(T) * 4);
+  L.hist = off;
+  off = align_up(off + static_cast<size_t>(T) * kBins * 4);
+  L.row_flag = off;
+  off = align_up(off + static_cast<size_t>(T));
+  L.block_flag = off;
+  off = align_up(off + static_cast<size_t>(L.n_blocks) * 4);
+  L.zero_end = off;
+  L.smin = off;
+  off = align_up(off + static_cast<size_t>(T) * 4);
+  L.width = off;
+  off = align_up(off + static_cast<size_t>(T) * 4);
+  L.thr = off;
+  off = align_up(off + static_cast<size_t>(T) * 4);
+  L.fb_list = off;
+  off = align_up(off + static_cast<size_t>(L.n_blocks) * 4);
+  // sample: keys every chunk row can see, i.e. positions 0 .. causal_offset, strided
+  long long prefix = static_cast<long long>(causal_offset) + 1;
+  if (prefix > N) prefix = N;
+  if (prefix < 0) prefix = 0;
+  long long want = static_cast<long long>(tun.sample_mult) * topk;
+  L.n_sample = static_cast<int>(want < prefix ? want : prefix);
+  L.sample_stride = L.n_sample > 0 ? static_cast<int>(prefix / L.n_sample) : 1;
+  L.sample = off;
+  off = align_up(off + static_cast<size_t>(T) * (L.n_sample > 0 ? L.n_sample : 1) * 4);
+  long long cap = static_cast<long long>(tun.cap_mult) * topk;
+  L.cap = static_cast<int>(cap > N ? N : cap);
+  L.cand = off;
+  off = align_up(off + static_cast<size_t>(T) * L.cap * 8);
+  size_t slot_bytes = static_cast<size_t>(kRowsPerBlock) * N * 4;
+  long long slots = static_cast<long long>(kFallbackScratchBudget / slot_bytes);
+  L.fb_slots = static_cast<int>(slots < 1 ? 1 : (slots > L.n_blocks ? L.n_blocks : slots));
+  L.scratch = off;
+  off = align_up(off + static_cast<size_t>(L.fb_slots) * slot_bytes);
+  L.total = off;
+  return L;
+}
+
+int sm_count() {
+  static int cached[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
+int pick_seg_tiles(const Tun& tun, int n_keys, int n_blocks, int grid) {
+  if (tun.segment_tiles > 0) return tun.segment_tiles;
+  int n_tiles = (n_keys + kTileKeys - 1) / kTileKeys;
+  int seg = 256;
+  while (seg > 16 && static_cast<long long>(n_blocks) * ((n_tiles + seg - 1) / seg) < 2ll * grid) seg >>= 1;
+  return seg;
+}
+
+// Control block for entry points that have no workspace (lt_indexer_scores).
+__device__ Control g_scores_ctl;
+
+// ---- the generic path: dense scores of a few rows at a time, then a full-row select ----------
+int run_unfused(int dtype, bool mma, const void* q, const float* w, const void* k, const float* k_scale, int T, int N, int H,
+                int D, int topk, int causal_offset, int32_t* out_idx, float* out_score, float* scores, int rows_per_pass,
+                Control* ctl, const Tun& tun, cudaStream_t stream) {
+  const int grid = tun.grid > 0 ? tun.grid : sm_count();
+  for (int r0 = 0; r0 < T; r0 += rows_per_pass) {
+    const int r1 = (r0 + rows_per_pass < T) ? r0 + rows_per_pass : T;
+    if (mma) {
+      ScanParams p{};
+      p.w = w;
+      p.k_scale = k_scale;
+      p.ks_stride = 1;
+      p.T = T;
+      p.row_begin = r0;
+      p.row_end = r1;
+      p.n_keys = N;
+      p.causal_offset = causal_offset;
+      p.skip_masked_tiles = 0;
+      p.seg_tiles = pick_seg_tiles(tun, N, (r1 - r0 + kRowsPerBlock - 1) / kRowsPerBlock, grid);
+      p.topk = topk;
+      p.dump = scores;
+      p.dump_ld = N;
+      p.ctl = ctl;
+      LT_CUDA(launch_scan_mma(dtype, kModeDump, q, T, k, N, D, p, grid, stream));
+    } else {
+      LT_CUDA(launch_simt_scores(dtype, q, w, k, k_scale, T, N, H, D, causal_offset, r0, r1, scores, N, stream));
+    }
+    if (topk > 0) {
+      SelectRowsParams sp{};
+      sp.scores = scores;
+      sp.ld = N;
+      sp.n_blocks = r1 - r0;
+      sp.row_begin = r0;
+      sp.T = T;
+      sp.N = N;
+      sp.topk = topk;
+      sp.causal_offset = causal_offset;
+      sp.out_idx = out_idx;
+      sp.out_score = out_score;
+      sp.ctl = ctl;
+      LT_CUDA(launch_select_rows(sp, stream));
+    }
+  }
+  return LT_OK;
+}
+
+int topk_impl(int dtype, const void* q, const float* w, const void* k, const float* k_scale, int T, int N, int H, int D, int topk,
+              int causal_offset, int32_t* out_idx, float* out_score, void* workspace, size_t workspace_bytes,
+              const lt_tunables* tunables, cudaStream_t stream) {
+  int rc = check_problem(dtype, q, w, k, k_scale, T, N, H, D);
+  if (rc != LT_OK) return rc;
+  if (out_idx == nullptr || topk <= 0 || topk > N || topk > LT_MAX_TOPK) return LT_ERR_INVALID_ARG;
+  const Tun tun = resolve_tunables(tunables);
+  const bool fused = use_fused(tun, dtype, H, D);
+  if (tun.path == LT_PATH_FUSED && !fused) return LT_ERR_UNSUPPORTED;
+  const Layout L = make_layout(fused, T, N, topk, causal_offset, tun);
+  if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) != 0 || workspace_bytes < L.total)
+    return LT_ERR_WORKSPACE;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  Control* ctl = reinterpret_cast<Control*>(ws + L.ctl);
+  LT_CUDA(cudaMemsetAsync(ws, 0, L.zero_end, stream));
+
+  if (!fused) {
+    return run_unfused(dtype, false, q, w, k, k_scale, T, N, H, D, topk, causal_offset, out_idx, out_score,
+                       reinterpret_cast<float*>(ws + L.scratch), L.generic_rows, ctl, tun, stream);
+  }
+
+  const int grid = tun.grid > 0 ? tun.grid : sm_count();
+  float* smin = reinterpret_cast<float*>(ws + L.smin);
+  float* width = reinterpret_cast<float*>(ws + L.width);
+  float* thr = reinterpret_cast<float*>(ws + L.thr);
+  unsigned int* tail = reinterpret_cast<unsigned int*>(ws + L.tail);
+  unsigned int* hist = reinterpret_cast<unsigned int*>(ws + L.hist);
+  unsigned char* row_flag = ws + L.row_flag;
+  unsigned int* block_flag = reinterpret_cast<unsigned int*>(ws + L.block_flag);
+  int* fb_list = reinterpret_cast<int*>(ws + L.fb_list);
+  float* sample = reinterpret_cast<float*>(ws + L.sample);
+  uint2* cand = reinterpret_cast<uint2*>(ws + L.cand);
+  float* scratch = reinterpret_cast<float*>(ws + L.scratch);
+
+  // 1. sample phase: score n_sample strided keys of the common prefix with the same tensor-core path
+  if (L.n_sample > 0) {
+    ScanParams p{};
+    p.w = w;
+    p.k_scale = k_scale;
+    p.ks_stride = L.sample_stride;
+    p.T = T;
+    p.row_begin = 0;
+    p.row_end = T;
+    p.n_keys = L.n_sample;
+    p.causal_offset = INT_MAX / 2;
+    p.skip_masked_tiles = 0;
+    p.seg_tiles = pick_seg_tiles(tun, L.n_sample, L.n_blocks, grid);
+    p.topk = topk;
+    p.dump = sample;
+    p.dump_ld = L.n_sample;
+    p.ctl = ctl;
+    LT_CUDA(launch_scan_mma(dtype, kModeDump, q, T, k, L.n_sample, static_cast<long long>(L.sample_stride) * D, p, grid, stream));
+  }
+  LT_CUDA(launch_sample_stats(sample, T, L.n_sample, topk, smin, width, thr, stream));
+
+  // 2. fused scan: score, gate, compact, count
+  {
+    ScanParams p{};
+    p.w = w;
+    p.k_scale = k_scale;
+    p.ks_stride = 1;
+    p.T = T;
+    p.row_begin = 0;
+    p.row_end = T;
+    p.n_keys = N;
+    p.causal_offset = causal_offset;
+    p.skip_masked_tiles = 1;
+    p.seg_tiles = pick_seg_tiles(tun, N, L.n_blocks, grid);
+    p.topk = topk;
+    p.thr = thr;
+    p.smin = smin;
+    p.width = width;
+    p.tail = tail;
+    p.hist = hist;
+    p.cand = cand;
+    p.cap = L.cap;
+    p.ctl = ctl;
+    LT_CUDA(launch_scan_mma(dtype, kModeFilter, q, T, k, N, D, p, grid, stream));
+  }
+
+  // 3. final select over the survivors; rows it cannot finish exactly are flagged
+  {
+    FinalSelectParams p{};
+    p.tail = tail;
+    p.hist = hist;
+    p.cand = cand;
+    p.smin = smin;
+    p.width = width;
+    p.cap = L.cap;
+    p.T = T;
+    p.N = N;
+    p.topk = topk;
+    p.causal_offset = causal_offset;
+    p.out_idx = out_idx;
+    p.out_score = out_score;
+    p.row_flag = row_flag;
+    p.block_flag = block_flag;
+    p.fb_list = fb_list;
+    p.ctl = ctl;
+    LT_CUDA(launch_final_select(p, stream));
+  }
+
+  // 4. exact fallback for flagged rows.  The host does not know how many there are, so it
+  // enqueues enough rounds for all blocks; rounds with nothing to do exit at once.
+  const int rounds = (L.n_blocks + L.fb_slots - 1) / L.fb_slots;
+  for (int r = 0; r < rounds; ++r) {
+    ScanParams p{};
+    p.w = w;
+    p.k_scale = k_scale;
+    p.ks_stride = 1;
+    p.T = T;
+    p.row_begin = 0;
+    p.row_end = T;
+    p.n_keys = N;
+    p.causal_offset = causal_offset;
+    p.skip_masked_tiles = 0;
+    p.seg_tiles = pick_seg_tiles(tun, N, L.fb_slots, grid);
+    p.topk = topk;
+    p.dump = scratch;
+    p.dump_ld = N;
+    p.fb_list = fb_list;
+    p.fb_blocks = &ctl->fb_blocks;
+    p.fb_round_base = r * L.fb_slots;
+    p.fb_slots = L.fb_slots;
+    p.ctl = ctl;
+    LT_CUDA(launch_scan_mma(dtype, kModeDump, q, T, k, N, D, p, grid, stream));
+    SelectRowsParams sp{};
+    sp.scores = scratch;
+    sp.ld = N;
+    sp.n_blocks = L.fb_slots * kRowsPerBlock;
+    sp.T = T;
+    sp.N = N;
+    sp.topk = topk;
+    sp.causal_offset = causal_offset;
+    sp.out_idx = out_idx;
+    sp.out_score = out_score;
+    sp.fb_list = fb_list;
+    sp.fb_blocks = &ctl->fb_blocks;
+    sp.fb_round_base = r * L.fb_slots;
+    sp.row_flag = row_flag;
+    sp.ctl = ctl;
+    LT_CUDA(launch_select_rows(sp, stream));
+  }
+  return LT_OK;
+}
+
+// ---- library-owned workspace of the 13-argument entry point -----------------------------------
+std::mutex g_arena_mu;
+void* g_arena = nullptr;
+size_t g_arena_bytes = 0;
+int g_arena_dev = -1;
+
+}  // namespace
+}  // namespace lt
+
+using namespace lt;
+
+extern "C" {
+
+int lt_version(void) { return LT_VERSION; }
+
+const char* lt_strerror(int code) {
+  switch (code) {
+    case LT_OK: return "ok";
+    case LT_ERR_INVALID_ARG: return "invalid argument";
+    case LT_ERR_UNSUPPORTED: return "unsupported dtype or shape";
+    case LT_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case LT_ERR_CUDA: return "CUDA runtime error";
+    default: return "unknown error code";
+  }
+}
+
+int lt_last_cuda_error(void) { return g_last_cuda_error; }
+
+size_t lt_indexer_topk_workspace_bytes(int dtype, int T, int N, int H, int D, int topk, const lt_tunables* tunables) {
+  if ((dtype != LT_DTYPE_F32 && dtype != LT_DTYPE_BF16 && dtype != LT_DTYPE_E4M3) || T <= 0 || N <= 0 || H <= 0 || D <= 0 ||
+      topk <= 0 || topk > N || topk > LT_MAX_TOPK)
+    return 0;
+  const Tun tun = resolve_tunables(tunables);
+  // the sample can never be larger with a different causal_offset than with the whole context visible
+  return make_layout(use_fused(tun, dtype, H, D), T, N, topk, N - 1, tun).total;
+}
+
+int lt_indexer_topk_ex(int dtype, const void* q, const float* w, const void* k, const float* k_scale, int T, int N, int H, int D,
+                       int topk, int causal_offset, int32_t* out_idx, float* out_score, void* workspace, size_t workspace_bytes,
+                       const lt_tunables* tunables, void* stream) {
+  return topk_impl(dtype, q, w, k, k_scale, T, N, H, D, topk, causal_offset, out_idx, out_score, workspace, workspace_bytes,
+                   tunables, static_cast<cudaStream_t>(stream));
+}
+
+int lt_indexer_topk(const void* q, const float* w, const void* k, const float* k_scale, int T, int N, int H, int D, int topk,
+                    int causal_offset, int32_t* out_idx, float* out_score, void* stream) {
+  const int dtype = (k_scale != nullptr) ? LT_DTYPE_E4M3 : LT_DTYPE_BF16;
+  int rc = check_problem(dtype, q, w, k, k_scale, T, N, H, D);
+  if (rc != LT_OK) return rc;
+  if (out_idx == nullptr || topk <= 0 || topk > N || topk > LT_MAX_TOPK) return LT_ERR_INVALID_ARG;
+  const size_t need = lt_indexer_topk_workspace_bytes(dtype, T, N, H, D, topk, nullptr);
+  if (need == 0) return LT_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_arena_mu);
+  int dev = 0;
+  LT_CUDA(cudaGetDevice(&dev));
+  if (g_arena == nullptr || g_arena_bytes < need || g_arena_dev != dev) {
+    if (g_arena != nullptr) {
+      LT_CUDA(cudaDeviceSynchronize());
+      cudaFree(g_arena);
+      g_arena = nullptr;
+      g_arena_bytes = 0;
+    }
+    LT_CUDA(cudaMalloc(&g_arena, need));
+    g_arena_bytes = need;
+    g_arena_dev = dev;
+  }
+  return topk_impl(dtype, q, w, k, k_scale, T, N, H, D, topk, causal_offset, out_idx, out_score, g_arena, g_arena_bytes, nullptr,
+                   static_cast<cudaStream_t>(stream));
+}
+
+int lt_indexer_scores(int dtype, const void* q, const float* w, const void* k, const float* k_scale, int T, int N, int H, int D,
+                      int causal_offset, int row_begin, int row_end, float* out_scores, int path, void* stream_) {
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  int rc = check_problem(dtype, q, w, k, k_scale, T, N, H, D);
+  if (rc != LT_OK) return rc;
+  if (out_scores == nullptr || row_begin < 0 || row_end > T || row_begin > row_end) return LT_ERR_INVALID_ARG;
+  if (row_begin == row_end) return LT_OK;
+  Tun tun = resolve_tunables(nullptr);
+  tun.path = path;
+  const bool mma = use_fused(tun, dtype, H, D);
+  if (path == LT_PATH_FUSED && !mma) return LT_ERR_UNSUPPORTED;
+  Control* ctl = nullptr;
+  LT_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&ctl), g_scores_ctl));
+  // run_unfused with topk == 0 only dumps; rows are written straight to the caller's matrix
+  const float* kk = k_scale;
+  int rows = row_end - row_begin;
+  if (mma) {
+    // the scan kernel addresses dump rows relative to row_begin
+    ScanParams p{};
+    const int grid = sm_count();
+    p.w = w;
+    p.k_scale = kk;
+    p.ks_stride = 1;
+    p.T = T;
+    p.row_begin = row_begin;
+    p.row_end = row_end;
+    p.n_keys = N;
+    p.causal_offset = causal_offset;
+    p.skip_masked_tiles = 0;
+    p.seg_tiles = pick_seg_tiles(tun, N, (rows + kRowsPerBlock - 1) / kRowsPerBlock, grid);
+    p.dump = out_scores;
+    p.dump_ld = N;
+    p.ctl = ctl;
+    LT_CUDA(launch_scan_mma(dtype, kModeDump, q, T, k, N, D, p, grid, stream));
+  } else {
+    LT_CUDA(launch_simt_scores(dtype, q, w, k, kk, T, N, H, D, causal_offset, row_begin, row_end, out_scores, N, stream));
+  }
+  return LT_OK;
+}
+
+int lt_unfused_topk(int dtype, const void* q, const float* w, const void* k, const float* k_scale, int T, int N, int H, int D,
+                    int topk, int causal_offset, int32_t* out_idx, float* out_score, float* score_buf, size_t score_buf_bytes,
+                    int path, void* stream_) {
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  int rc = check_problem(dtype, q, w, k, k_scale, T, N, H, D);
+  if (rc != LT_OK) return rc;
+  if (out_idx == nullptr || topk <= 0 || topk > N || topk > LT_MAX_TOPK) return LT_ERR_INVALID_ARG;
+  if (score_buf == nullptr || (reinterpret_cast<uintptr_t>(score_buf) & (kAlign - 1)) != 0) return LT_ERR_WORKSPACE;
+  Tun tun = resolve_tunables(nullptr);
+  tun.path = path;
+  const bool mma = use_fused(tun, dtype, H, D);
+  if (path == LT_PATH_FUSED && !mma) return LT_ERR_UNSUPPORTED;
+  // the first 256 bytes of score_buf hold the status block (readable with lt_read_status)
+  if (score_buf_bytes < kAlign + static_cast<size_t>(N) * 4) return LT_ERR_WORKSPACE;
+  long long rows = static_cast<long long>((score_buf_bytes - kAlign) / (static_cast<size_t>(N) * 4));
+  if (rows > T) rows = T;
+  if (mma && rows >= kRowsPerBlock) rows -= rows % kRowsPerBlock;
+  Control* ctl = reinterpret_cast<Control*>(score_buf);
+  LT_CUDA(cudaMemsetAsync(ctl, 0, kAlign, stream));
+  float* scores = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(score_buf) + kAlign);
+  return run_unfused(dtype, mma, q, w, k, k_scale, T, N, H, D, topk, causal_offset, out_idx, out_score, scores,
+                     static_cast<int>(rows), ctl, tun, stream);
+}
+
+int lt_read_status(const void* workspace, int* status8_host, void* stream) {
+  if (status8_host == nullptr) return LT_ERR_INVALID_ARG;
+  const void* src = workspace;
+  if (src == nullptr) {
+    std::lock_guard<std::mutex> lock(g_arena_mu);
+    src = g_arena;
+  }
+  if (src == nullptr) return LT_ERR_WORKSPACE;
+  LT_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+  LT_CUDA(cudaMemcpy(status8_host, src, 8 * sizeof(int), cudaMemcpyDeviceToHost));
+  return LT_OK;
+}
+
+void lt_shutdown(void) {
+  std::lock_guard<std::mutex> lock(g_arena_mu);
+  if (g_arena != nullptr) {
+    cudaDeviceSynchronize();
+    cudaFree(g_arena);
+    g_arena = nullptr;
+    g_arena_bytes = 0;
+    g_arena_dev = -1;
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,102 @@
+// Host-side declarations shared by the library's translation units (not part of the public ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "lt_common.cuh"
+
+namespace lt {
+
+constexpr int kModeFilter = 0;
+constexpr int kModeDump = 1;
+constexpr int kRowsPerBlock = 8;  // query rows one scan CTA keeps resident
+
+// Parameters of the tensor-core scan kernel (lt_scan_mma.cu).
+struct ScanParams {
+  const float* w;          // [T][64]
+  const float* k_scale;    // per key of the view, or null
+  long long ks_stride;     // k_scale index of view key s is s * ks_stride
+  int T;                   // rows of q / w
+  int row_begin, row_end;  // rows handled by this launch (ignored when fb_list is set)
+  int n_keys;              // keys in the view
+  int causal_offset;       // row t sees view keys 0 .. causal_offset + t
+  int skip_masked_tiles;   // 1: do not visit key tiles no row of the block can see
+  int seg_tiles;           // key tiles per work item
+  int topk;
+  // filter mode
+  float* thr;              // [T] gate: lower edge of the row's threshold bin (-inf = accept all)
+  const float* smin;       // [T] sampled minimum score
+  const float* width;      // [T] bin width
+  unsigned int* tail;      // [T] survivors appended so far (may exceed cap)
+  unsigned int* hist;      // [T][kBins]
+  uint2* cand;             // [T][cap] (score bits, key index)
+  int cap;
+  // dump mode
+  float* dump;             // dense scores
+  long long dump_ld;       // row pitch of dump in floats
+  // exact-fallback dump: blocks come from a device-side list, slot j of this round
+  // is block fb_list[fb_round_base + j], its rows go to dump rows 8j .. 8j+7
+  const int* fb_list;
+  const int* fb_blocks;    // device counter: entries in fb_list
+  int fb_round_base;
+  int fb_slots;
+  Control* ctl;
+};
+
+bool scan_mma_supported(int dtype, int H, int D);
+
+// q: [T][64][128]; k: view of n_keys_view rows whose pitch is key_pitch_elems elements.
+cudaError_t launch_scan_mma(int dtype, int mode, const void* q, int T, const void* k, long long n_keys_view,
+                            long long key_pitch_elems, const ScanParams& p, int grid, cudaStream_t stream);
+
+// ---- lt_select.cu ---------------------------------------------------------------------------
+// Generic SIMT scoring (any H, D, dtype): dense scores of rows [row_begin, row_end), -inf where masked.
+cudaError_t launch_simt_scores(int dtype, const void* q, const float* w, const void* k, const float* k_scale, int T, int N,
+                               int H, int D, int causal_offset, int row_begin, int row_end, float* out, long long ld,
+                               cudaStream_t stream);
+
+// Sample statistics (paper Sec. 3.2 "Sampling"): per row min / max of the sampled scores, bin
+// width, and the threshold edge of the bin holding the k-th largest sampled score.
+cudaError_t launch_sample_stats(const float* sample, int T, int n_sample, int topk, float* smin, float* width, float* thr,
+                                cudaStream_t stream);
+
+// Final selection from the candidate buffers (paper Sec. 3.2 "Top-k Selection"); rows that cannot
+// be finished exactly are flagged and their block appended to the fallback list.
+struct FinalSelectParams {
+  const unsigned int* tail;
+  const unsigned int* hist;
+  const uint2* cand;
+  const float* smin;
+  const float* width;
+  int cap, T, N, topk, causal_offset;
+  int32_t* out_idx;
+  float* out_score;
+  unsigned char* row_flag;    // [T] 1 = needs the fallback
+  unsigned int* block_flag;   // [ceil(T/8)]
+  int* fb_list;               // [ceil(T/8)]
+  Control* ctl;
+};
+cudaError_t launch_final_select(const FinalSelectParams& p, cudaStream_t stream);
+
+// Full-row exact select over dense scores.  Direct mode: block b handles row row_begin + b whose
+// scores start at scores + b * ld.  Fallback mode (fb_list != null): block b handles row
+// fb_list[fb_round_base + b / 8] * 8 + b % 8 if that row is flagged; scores at scores + b * ld.
+struct SelectRowsParams {
+  const float* scores;
+  long long ld;
+  int n_blocks;  // CTAs to launch
+  int row_begin;
+  int T, N, topk, causal_offset;
+  int32_t* out_idx;
+  float* out_score;
+  const int* fb_list;
+  const int* fb_blocks;
+  int fb_round_base;
+  const unsigned char* row_flag;
+  Control* ctl;
+};
+cudaError_t launch_select_rows(const SelectRowsParams& p, cudaStream_t stream);
+
+}  // namespace lt

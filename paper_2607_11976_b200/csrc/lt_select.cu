@@ -1,0 +1,360 @@
+// Selection-side kernels of the indexer top-k: sample statistics, final select over the candidate
+// buffers, full-row radix select (generic path, unfused baseline, exact fallback) and the generic
+// SIMT scoring kernel.
+#include <cuda_bf16.h>
+#include <cuda_fp8.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+
+#include "lt_common.cuh"
+#include "lt_host.h"
+
+namespace lt {
+
+namespace {
+
+constexpr int kSelThreads = 1024;
+constexpr int kSelCap = 2 * LT_MAX_TOPK;  // 64-bit keys the final select can sort in shared memory
+
+// ---------------------------------------------------------------------------------------------
+// generic SIMT scoring: one CTA = one query row x 128 keys; thread = one key.
+// ---------------------------------------------------------------------------------------------
+template <int kDtype>
+__device__ __forceinline__ float load_elem(const void* base, size_t i) {
+  if (kDtype == LT_DTYPE_F32) return reinterpret_cast<const float*>(base)[i];
+  if (kDtype == LT_DTYPE_BF16) return __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const uint16_t*>(base)[i]) << 16);
+  __half_raw hr = __nv_cvt_fp8_to_halfraw(reinterpret_cast<const uint8_t*>(base)[i], __NV_E4M3);
+  return __half2float(__half(hr));
+}
+
+template <int kDtype>
+__global__ void __launch_bounds__(128) simt_scores_kernel(const void* __restrict__ q, const float* __restrict__ w,
+                                                          const void* __restrict__ k, const float* __restrict__ k_scale, int N,
+                                                          int H, int D, int causal_offset, int row_begin, float* __restrict__ out,
+                                                          long long ld) {
+  extern __shared__ float sm[];
+  float* qs = sm;                 // [H][D]
+  float* ks = sm + H * D;         // [128][D + 1]
+  const int t = row_begin + blockIdx.y;
+  const int s0 = blockIdx.x * 128;
+  for (int i = threadIdx.x; i < H * D; i += 128) qs[i] = load_elem<kDtype>(q, static_cast<size_t>(t) * H * D + i);
+  for (int i = threadIdx.x; i < 128 * D; i += 128) {
+    int r = i / D, d = i - r * D;
+    int s = s0 + r;
+    ks[r * (D + 1) + d] = (s < N) ? load_elem<kDtype>(k, static_cast<size_t>(s) * D + d) : 0.f;
+  }
+  __syncthreads();
+  const int s = s0 + threadIdx.x;
+  if (s >= N) return;
+  const float* kr = ks + threadIdx.x * (D + 1);
+  float total = 0.f;
+  for (int h = 0; h < H; ++h) {
+    const float* qh = qs + h * D;
+    float dot = 0.f;
+    for (int d = 0; d < D; ++d) dot = __fmaf_rn(qh[d], kr[d], dot);
+    total = __fmaf_rn(w[static_cast<size_t>(t) * H + h], fmaxf(dot, 0.f), total);
+  }
+  if (k_scale != nullptr) total *= k_scale[s];
+  total += 0.f;  // -0 -> +0
+  const int vis = visible_keys(t, N, causal_offset);
+  out[static_cast<size_t>(blockIdx.y) * ld + s] = (s < vis) ? total : -INFINITY;
+}
+
+// ---------------------------------------------------------------------------------------------
+// sample statistics: one CTA per row.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) sample_stats_kernel(const float* __restrict__ sample, int n_sample, int topk,
+                                                           float* __restrict__ smin_out, float* __restrict__ width_out,
+                                                           float* __restrict__ thr_out) {
+  __shared__ float red_min[8], red_max[8];
+  __shared__ unsigned int hist[kBins];
+  __shared__ float s_min, s_width;
+  const int t = blockIdx.x;
+  const float* row = sample + static_cast<size_t>(t) * n_sample;
+  float mn = INFINITY, mx = -INFINITY;
+  for (int i = threadIdx.x; i < n_sample; i += 256) {
+    float v = row[i];
+    mn = fminf(mn, v);
+    mx = fmaxf(mx, v);
+  }
+  for (int d = 16; d > 0; d >>= 1) {
+    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, d));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
+  }
+  if ((threadIdx.x & 31) == 0) {
+    red_min[threadIdx.x >> 5] = mn;
+    red_max[threadIdx.x >> 5] = mx;
+  }
+  hist[threadIdx.x] = 0;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int i = 1; i < 8; ++i) {
+      mn = fminf(mn, red_min[i]);
+      mx = fmaxf(mx, red_max[i]);
+    }
+    if (n_sample <= 0) mn = mx = 0.f;
+    s_min = mn;
+    s_width = (mx - mn) / static_cast<float>(kBins);
+  }
+  __syncthreads();
+  const float smin = s_min, width = s_width;
+  for (int i = threadIdx.x; i < n_sample; i += 256) atomicAdd(&hist[bin_of(row[i], smin, width)], 1u);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    // threshold bin = bin holding the k-th largest sampled score; 0 (accept all) if the sample is smaller than k
+    int tb = 0;
+    unsigned int cum = 0;
+    for (int b = kBins - 1; b >= 1; --b) {
+      cum += hist[b];
+      if (cum >= static_cast<unsigned int>(topk)) {
+        tb = b;
+        break;
+      }
+    }
+    smin_out[t] = smin;
+    width_out[t] = width;
+    thr_out[t] = bin_edge(tb, smin, width);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// sort the first `count` keys of sel[] (shared) and write the row's outputs.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void sort_and_write(uint64_t* sel, int count, int topk, int32_t* out_idx, float* out_score) {
+  const int n = next_pow2(count < 2 ? 2 : count);
+  for (int i = count + threadIdx.x; i < n; i += blockDim.x) sel[i] = 0ull;
+  __syncthreads();
+  bitonic_sort_desc(sel, n, threadIdx.x, blockDim.x);
+  for (int j = threadIdx.x; j < topk; j += blockDim.x) {
+    bool have = j < count;
+    out_idx[j] = have ? key_index(sel[j]) : -1;
+    if (out_score != nullptr) out_score[j] = have ? key_score(sel[j]) : -INFINITY;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// final select over one row's candidate buffer.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kSelThreads) final_select_kernel(const FinalSelectParams p) {
+  extern __shared__ uint64_t sel[];  // kSelCap keys
+  __shared__ unsigned int hist[kBins];
+  __shared__ int s_tb;
+  __shared__ unsigned int s_count;
+  const int t = blockIdx.x;
+  const unsigned int tail = p.tail[t];
+  const int vis = visible_keys(t, p.N, p.causal_offset);
+  const int kk = p.topk < vis ? p.topk : vis;
+  bool redo = tail > static_cast<unsigned int>(p.cap);
+  if (threadIdx.x == 0) {
+    atomicMax(&p.ctl->max_survivors, static_cast<int>(tail > 0x7fffffffu ? 0x7fffffffu : tail));
+    atomicAdd(&p.ctl->tot_survivors, static_cast<int>(tail > 0x000fffffu ? 0x000fffffu : tail));
+    if (redo) atomicAdd(&p.ctl->overflow_rows, 1);
+  }
+  if (!redo) {
+    if (threadIdx.x < kBins) hist[threadIdx.x] = p.hist[static_cast<size_t>(t) * kBins + threadIdx.x];
+    if (threadIdx.x == 0) s_count = 0;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      // final threshold bin: the bins above it hold fewer than k candidates
+      int tb = 0;
+      unsigned int cum = 0;
+      for (int b = kBins - 1; b >= 1; --b) {
+        cum += hist[b];
+        if (cum >= static_cast<unsigned int>(kk)) {
+          tb = b;
+          break;
+        }
+      }
+      s_tb = tb;
+    }
+    __syncthreads();
+    const float edge = bin_edge(s_tb, p.smin[t], p.width[t]);
+    const uint2* cand = p.cand + static_cast<size_t>(t) * p.cap;
+    for (unsigned int i = threadIdx.x; i < tail; i += kSelThreads) {
+      uint2 c = cand[i];
+      float sc = __uint_as_float(c.x);
+      if (sc >= edge) {
+        unsigned int pos = atomicAdd(&s_count, 1u);
+        if (pos < static_cast<unsigned int>(kSelCap)) sel[pos] = pack_key(sc, static_cast<int>(c.y));
+      }
+    }
+    __syncthreads();
+    const unsigned int count = s_count;
+    // count < kk cannot happen for an exact filter; treating it as "redo" keeps the result exact regardless
+    if (count > static_cast<unsigned int>(kSelCap) || count < static_cast<unsigned int>(kk)) redo = true;
+    if (!redo) {
+      sort_and_write(sel, static_cast<int>(count), p.topk, p.out_idx + static_cast<size_t>(t) * p.topk,
+                     p.out_score ? p.out_score + static_cast<size_t>(t) * p.topk : nullptr);
+      return;
+    }
+  }
+  if (threadIdx.x == 0) {
+    p.row_flag[t] = 1;
+    atomicOr(&p.ctl->status, LT_STATUS_FALLBACK);
+    atomicAdd(&p.ctl->fb_rows, 1);
+    if (atomicExch(p.block_flag + t / kRowsPerBlock, 1u) == 0u) {
+      int pos = atomicAdd(&p.ctl->fb_blocks, 1);
+      p.fb_list[pos] = t / kRowsPerBlock;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// full-row exact select: 4-pass MSB radix select for the k-th key, ordered collection of ties
+// (lowest indices first), bitonic sort of the k winners.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kSelThreads) select_rows_kernel(const SelectRowsParams p) {
+  extern __shared__ uint64_t sel[];  // LT_MAX_TOPK keys
+  __shared__ unsigned int hist[256];
+  __shared__ unsigned int s_prefix, s_remaining, s_gt, s_eq_base;
+  __shared__ unsigned int warp_cnt[32];
+  int t;
+  if (p.fb_list != nullptr) {
+    int j = p.fb_round_base + blockIdx.x / kRowsPerBlock;
+    if (j >= *p.fb_blocks) return;
+    t = p.fb_list[j] * kRowsPerBlock + blockIdx.x % kRowsPerBlock;
+    if (t >= p.T || !p.row_flag[t]) return;
+  } else {
+    t = p.row_begin + blockIdx.x;
+  }
+  const float* row = p.scores + static_cast<size_t>(blockIdx.x) * p.ld;
+  const int vis = visible_keys(t, p.N, p.causal_offset);
+  const int kk = p.topk < vis ? p.topk : vis;
+  int32_t* out_idx = p.out_idx + static_cast<size_t>(t) * p.topk;
+  float* out_score = p.out_score ? p.out_score + static_cast<size_t>(t) * p.topk : nullptr;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+
+  if (vis <= p.topk) {
+    // every visible key is selected
+    for (int i = tid; i < vis; i += kSelThreads) sel[i] = pack_key(row[i], i);
+    __syncthreads();
+    sort_and_write(sel, vis, p.topk, out_idx, out_score);
+    return;
+  }
+
+  if (tid == 0) {
+    s_prefix = 0;
+    s_remaining = static_cast<unsigned int>(kk);
+  }
+  unsigned int mask = 0;
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    if (tid < 256) hist[tid] = 0;
+    __syncthreads();
+    const unsigned int prefix = s_prefix;
+    for (int i = tid; i < vis; i += kSelThreads) {
+      unsigned int key = score_to_key(__float_as_uint(row[i]));
+      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (tid == 0) {
+      unsigned int remaining = s_remaining, cum = 0;
+      int digit = 0;
+      for (int d = 255; d >= 0; --d) {
+        unsigned int c = hist[d];
+        if (cum + c >= remaining) {
+          digit = d;
+          break;
+        }
+        cum += c;
+      }
+      s_remaining = remaining - cum;  // still needed among keys that share the longer prefix
+      s_prefix = prefix | (static_cast<unsigned int>(digit) << shift);
+    }
+    mask |= 0xffu << shift;
+    __syncthreads();
+  }
+  const unsigned int kth = s_prefix;                 // key of the k-th largest score
+  const unsigned int need_eq = s_remaining;          // how many keys equal to it are selected
+  const unsigned int n_gt = static_cast<unsigned int>(kk) - need_eq;
+  if (tid == 0) {
+    s_gt = 0;
+    s_eq_base = 0;
+  }
+  __syncthreads();
+  for (int base = 0; base < vis; base += kSelThreads) {
+    const int i = base + tid;
+    unsigned int key = 0;
+    bool gt = false, eq = false;
+    if (i < vis) {
+      key = score_to_key(__float_as_uint(row[i]));
+      gt = key > kth;
+      eq = key == kth;
+    }
+    if (gt) {
+      unsigned int pos = atomicAdd(&s_gt, 1u);
+      sel[pos] = (static_cast<uint64_t>(key) << 32) | (0xffffffffu - static_cast<unsigned int>(i));
+    }
+    // ties at the k-th value: keep the lowest indices, so rank them in index order
+    const unsigned int eq_ballot = __ballot_sync(0xffffffffu, eq);
+    if (lane == 0) warp_cnt[wid] = __popc(eq_ballot);
+    __syncthreads();
+    const unsigned int eq_base = s_eq_base;
+    unsigned int before = 0, total = 0;
+    for (int wq = 0; wq < 32; ++wq) {
+      unsigned int c = warp_cnt[wq];
+      if (wq < wid) before += c;
+      total += c;
+    }
+    if (eq) {
+      unsigned int rank = eq_base + before + __popc(eq_ballot & ((1u << lane) - 1u));
+      if (rank < need_eq) sel[n_gt + rank] = (static_cast<uint64_t>(key) << 32) | (0xffffffffu - static_cast<unsigned int>(i));
+    }
+    __syncthreads();
+    if (tid == 0) s_eq_base = eq_base + total;
+    __syncthreads();
+  }
+  sort_and_write(sel, kk, p.topk, out_idx, out_score);
+}
+
+}  // namespace
+
+cudaError_t launch_simt_scores(int dtype, const void* q, const float* w, const void* k, const float* k_scale, int T, int N,
+                               int H, int D, int causal_offset, int row_begin, int row_end, float* out, long long ld,
+                               cudaStream_t stream) {
+  (void)T;
+  const int rows = row_end - row_begin;
+  if (rows <= 0) return cudaSuccess;
+  const size_t smem = (static_cast<size_t>(H) * D + 128 * (D + 1)) * sizeof(float);
+  dim3 grid((N + 127) / 128, rows);
+  cudaError_t e;
+#define LT_SIMT_CASE(DT)                                                                                              \
+  e = cudaFuncSetAttribute(simt_scores_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)); \
+  if (e != cudaSuccess) return e;                                                                                       \
+  simt_scores_kernel<DT><<<grid, 128, smem, stream>>>(q, w, k, k_scale, N, H, D, causal_offset, row_begin, out, ld);
+  if (dtype == LT_DTYPE_F32) {
+    LT_SIMT_CASE(LT_DTYPE_F32)
+  } else if (dtype == LT_DTYPE_BF16) {
+    LT_SIMT_CASE(LT_DTYPE_BF16)
+  } else {
+    LT_SIMT_CASE(LT_DTYPE_E4M3)
+  }
+#undef LT_SIMT_CASE
+  return cudaGetLastError();
+}
+
+cudaError_t launch_sample_stats(const float* sample, int T, int n_sample, int topk, float* smin, float* width, float* thr,
+                                cudaStream_t stream) {
+  sample_stats_kernel<<<T, 256, 0, stream>>>(sample, n_sample, topk, smin, width, thr);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_final_select(const FinalSelectParams& p, cudaStream_t stream) {
+  const int smem = kSelCap * sizeof(uint64_t);
+  cudaError_t e = cudaFuncSetAttribute(final_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  final_select_kernel<<<p.T, kSelThreads, smem, stream>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_select_rows(const SelectRowsParams& p, cudaStream_t stream) {
+  const int smem = LT_MAX_TOPK * sizeof(uint64_t);
+  cudaError_t e = cudaFuncSetAttribute(select_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  if (p.n_blocks <= 0) return cudaSuccess;
+  select_rows_kernel<<<p.n_blocks, kSelThreads, smem, stream>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace lt

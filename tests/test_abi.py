@@ -1,0 +1,82 @@
+"""The C-ABI library builds, loads, and exports every symbol the public header declares.
+No GPU is needed: only host-side argument checks are exercised."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2607_11976_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "lt_indexer.h")
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.load()
+
+
+def declared_functions():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(lt_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_header_symbols_exported(lib):
+    names = declared_functions()
+    assert {"lt_indexer_topk", "lt_indexer_topk_ex", "lt_indexer_scores", "lt_unfused_topk",
+            "lt_indexer_topk_workspace_bytes", "lt_read_status", "lt_strerror", "lt_version", "lt_shutdown"} <= set(names)
+    for name in names:
+        assert hasattr(lib, name), f"{name} declared in lt_indexer.h but not exported"
+
+
+def test_version_and_strerror(lib):
+    assert lib.lt_version() == 100
+    assert lib.lt_strerror(0) == b"ok"
+    assert b"invalid" in lib.lt_strerror(-1)
+    assert b"unknown" in lib.lt_strerror(-77)
+
+
+def test_host_side_argument_checks(lib):
+    null = ctypes.c_void_p(None)
+    fake = ctypes.c_void_p(0x1000)  # aligned, never dereferenced: the checks fail first
+    odd = ctypes.c_void_p(0x1004)
+    # null pointers
+    assert lib.lt_indexer_topk(null, fake, fake, null, 8, 64, 64, 128, 4, 56, fake, null, null) == -1
+    # topk > N and non-positive sizes
+    assert lib.lt_indexer_topk(fake, fake, fake, null, 8, 64, 64, 128, 65, 56, fake, null, null) == -1
+    assert lib.lt_indexer_topk(fake, fake, fake, null, 0, 64, 64, 128, 4, 56, fake, null, null) == -1
+    # misaligned q
+    assert lib.lt_indexer_topk(odd, fake, fake, null, 8, 64, 64, 128, 4, 56, fake, null, null) == -1
+    # unknown dtype, fp8 without scales
+    assert lib.lt_indexer_topk_ex(9, fake, fake, fake, null, 8, 64, 64, 128, 4, 56, fake, null, fake, 1 << 30, None, null) == -2
+    assert lib.lt_indexer_topk_ex(2, fake, fake, fake, null, 8, 64, 64, 128, 4, 56, fake, null, fake, 1 << 30, None, null) == -1
+    # workspace too small / missing
+    assert lib.lt_indexer_topk_ex(1, fake, fake, fake, null, 8, 64, 64, 128, 4, 56, fake, null, fake, 16, None, null) == -3
+    assert lib.lt_indexer_topk_ex(1, fake, fake, fake, null, 8, 64, 64, 128, 4, 56, fake, null, null, 0, None, null) == -3
+    # the fused path cannot be forced onto a shape it does not support
+    tun = binding.Tunables(path=binding.LT_PATH_FUSED)
+    assert lib.lt_indexer_topk_ex(0, fake, fake, fake, null, 8, 64, 8, 64, 4, 56, fake, null, fake, 1 << 30,
+                                  ctypes.byref(tun), null) == -2
+    assert lib.lt_indexer_scores(1, fake, fake, fake, null, 8, 64, 64, 128, 56, 3, 2, fake, 0, null) == -1
+    assert lib.lt_unfused_topk(1, fake, fake, fake, null, 8, 64, 64, 128, 4, 56, fake, null, null, 0, 0, null) == -3
+
+
+def test_workspace_arithmetic(lib):
+    # candidate buffer: 8192 rows x 12k (24,576) entries x 8 B = 1.5 GiB, the figure the paper's Sec. 4.2
+    # quotes for k = 2048; the total adds histograms, the sample scores and the fallback scratch
+    T, N, H, D, k = 8192, 1 << 20, 64, 128, 2048
+    total = binding.lt_indexer_topk_workspace_bytes("e4m3", T, N, H, D, k)
+    cand = T * 12 * k * 8
+    assert cand == 1536 << 20
+    assert cand < total < cand + (1 << 30)
+    half = binding.lt_indexer_topk_workspace_bytes("e4m3", T, N, H, D, k, binding.Tunables(cap_mult=6))
+    assert total - half == cand // 2
+    # invalid problems report 0
+    assert binding.lt_indexer_topk_workspace_bytes("bf16", 8, 64, 64, 128, 65) == 0
+    assert binding.lt_indexer_topk_workspace_bytes("bf16", 8, 64, 64, 128, 9000) == 0
+    # generic path: a bounded dense-score scratch
+    g = binding.lt_indexer_topk_workspace_bytes("f32", 64, 4096, 8, 64, 256)
+    assert 64 * 4096 * 4 <= g <= 64 * 4096 * 4 + 4096
