@@ -1,0 +1,365 @@
+#!/usr/bin/env python
+"""Benchmark of the fused DSA indexer top-k on B200.
+
+One "step" is one pass of the whole hot path (sample scoring, sample statistics, fused
+score + filter scan, final select, exact fallback rounds) over one synthetic chunk.  Default
+workload: `fp8_1m`, the last 4096-query chunk of a 1,048,576-token prefill (H = 64, D = 128,
+top-k = 2048, e4m3 codes with per-token fp32 scales), the configuration the headline metric is
+quoted on.  The metric is scored (query, key) pairs per second over the causally valid pairs.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+N > 1 (launched under torchrun) runs N independent replicas, one per GPU: the path has no exchange
+step, so there is no data-path collective; only the timing barrier and the max-over-ranks
+reduction go through NCCL.  `--impl reference` times the CPU oracle on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "scored_query_key_pairs_per_second"
+UNIT = "pairs/s"
+NOMINAL_FP8_TFLOPS = 4500.0
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM bytes of one launch of the fused scan kernel (dram__bytes_read.sum + dram__bytes_write.sum),
+# per scored pair, from the ncu capture summarised under profiles/; scaled by the pairs of a launch.
+SCAN_DRAM_BYTES_PER_PAIR = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.lines = []
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._pump, daemon=True)
+        self.thread.start()
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, power, reasons = [], [], [], set()
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+                power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        # the busiest samples are the ones under load
+        loaded = [c for c, p in zip(sm, power) if power and p >= 0.6 * max(power)] or sm
+        return {"sm_mhz": statistics.median(loaded) if loaded else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def cpu_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+
+        n = [p.get("num_threads", 0) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def time_oracle(inp, budget_s: float, max_rows: int = 64):
+    """Times the CPU oracle, as it stands, on a bounded sample of rows of the same workload:
+    evenly spaced rows (each against every key it may see), stopping once the budget is spent."""
+    from oracle import decode, oracle_topk
+
+    np.matmul(np.ones((64, 64)), np.ones((64, 64)))  # start the BLAS threads
+    rows = np.unique(np.linspace(0, inp.T - 1, max_rows).astype(np.int64))
+    t0 = time.perf_counter()
+    # the oracle decodes K on every call; do the sample in row batches so the budget can stop it
+    done_rows, pairs = 0, 0
+    batch = 4
+    for i in range(0, len(rows), batch):
+        chunk = rows[i:i + batch]
+        oracle_topk(inp, rows=chunk)
+        done_rows += len(chunk)
+        pairs += sum(inp.visible(int(t)) for t in chunk)
+        if time.perf_counter() - t0 > budget_s:
+            break
+    dt = time.perf_counter() - t0
+    return pairs / dt, done_rows, pairs, dt
+
+
+def run_reference(args, rank: int):
+    """`--impl reference`: the CPU oracle on the host cores, rank 0 only."""
+    if rank != 0:
+        return
+    from workloads import make_config
+
+    inp = make_config(args.workload)
+    steps_val = []
+    for _ in range(args.warmup):
+        time_oracle(inp, budget_s=1.0, max_rows=4)
+    sample = ""
+    for _ in range(args.steps):
+        v, rows, pairs, dt = time_oracle(inp, budget_s=args.cpu_budget / max(1, args.steps), max_rows=16)
+        steps_val.append((v, dt))
+        sample = f"{rows} evenly spaced rows x all visible keys ({pairs} pairs) per step"
+    value = statistics.mean(v for v, _ in steps_val)
+    ms = statistics.mean(dt for _, dt in steps_val) * 1e3
+    cores = cpu_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "T": inp.T, "N": inp.N, "H": inp.H, "D": inp.D, "topk": inp.topk,
+                   "note": "CPU oracle (numpy fp64 + full sort) on a bounded row sample of the workload"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="fp8_1m")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of CPU work for the oracle baseline")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-unfused", action="store_true")
+    ap.add_argument("--unfused-budget-mb", type=int, default=2048, help="score-matrix budget of the unfused GPU baseline")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_2607_11976_b200 import binding as lt
+    from paper_2607_11976_b200 import build as lt_build
+    from workloads import make_config
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    args.warmup = max(args.warmup, 3)
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        lt_build.build()
+    if world > 1:
+        dist.barrier()
+    lt.load()
+
+    inp = make_config(args.workload)
+    pairs = inp.valid_pairs()
+    flops = 2.0 * inp.H * inp.D * pairs
+    q, w, k, ks = lt.to_device(inp)
+    out_idx = torch.empty((inp.T, inp.topk), dtype=torch.int32, device="cuda")
+    out_score = torch.empty((inp.T, inp.topk), dtype=torch.float32, device="cuda")
+    ws = lt.alloc_workspace(inp.dtype, inp.T, inp.N, inp.H, inp.D, inp.topk)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")  # larger than the 126 MB L2
+    stream = torch.cuda.current_stream()
+
+    def step():
+        lt.lt_indexer_topk_ex(inp.dtype, q, w, k, ks, inp.topk, inp.causal_offset, out_idx, out_score, ws)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    lt.lt_set_profiling(True)
+    for _ in range(args.warmup):
+        step()
+    status = lt.lt_read_status(ws)
+    if status[0] & lt.LT_STATUS_TIMEOUT:
+        raise SystemExit("device-side wait timed out; results invalid")
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    barrier()
+    launches0 = lt.lt_launch_count()
+    step_ms, phase_ms = [], []
+    for _ in range(args.steps):
+        flush.fill_(1)  # evict L2 between timed iterations (untimed)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        step()
+        e1.record(stream)
+        e1.synchronize()
+        step_ms.append(e0.elapsed_time(e1))
+        phase_ms.append(lt.lt_read_phase_ms())
+    launches = lt.lt_launch_count() - launches0
+    barrier()
+    clocks = sampler.stop()
+    total_ms = sum(step_ms)
+    if world > 1:
+        tmax = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        total_ms = float(tmax.item())
+    ms_per_step = total_ms / args.steps
+    value = world * pairs * args.steps / (total_ms * 1e-3)
+    status = lt.lt_read_status(ws)
+
+    # ---- end to end through the public API with host buffers: H2D of the inputs, D2H of the result
+    host = [t.cpu().pin_memory() for t in (q, w, k)] + ([ks.cpu().pin_memory()] if ks is not None else [])
+    dev = [q, w, k] + ([ks] if ks is not None else [])
+    h_idx = torch.empty_like(out_idx, device="cpu").pin_memory()
+    h_score = torch.empty_like(out_score, device="cpu").pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in host)
+    d2h = h_idx.numel() * 4 + h_score.numel() * 4
+
+    def e2e_step():
+        for d, h in zip(dev, host):
+            d.copy_(h, non_blocking=True)
+        step()
+        h_idx.copy_(out_idx, non_blocking=True)
+        h_score.copy_(out_score, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e2e_steps = min(args.steps, 5)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    e1.synchronize()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        tmax = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tmax.item())
+    e2e_value = world * pairs * e2e_steps / (e2e_ms * 1e-3)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_kind = load_peaks()
+    fp8 = inp.dtype == "e4m3"
+    # measured dense peak for this dtype: the measured bf16 burst figure x the nominal fp8:bf16 ratio (2)
+    peak_tflops = peaks["bf16_tflops"] * (2.0 if fp8 else 1.0)
+    scan_ms = statistics.mean(p[2] for p in phase_ms)
+    achieved = flops / (scan_ms * 1e-3) / 1e12
+    roofline = {
+        "bound": "tensor", "kernel": "scan_kernel (fused score + filter)", "achieved": achieved, "peak": peak_tflops,
+        "unit": "TFLOP/s", "frac": achieved / peak_tflops, "peak_kind": f"of {peak_kind} (bf16 burst x {2 if fp8 else 1})",
+        "frac_of_nominal": achieved / (NOMINAL_FP8_TFLOPS if fp8 else NOMINAL_BF16_TFLOPS),
+        "flops_per_launch": flops, "kernel_ms": scan_ms,
+        "traffic": None if SCAN_DRAM_BYTES_PER_PAIR is None else SCAN_DRAM_BYTES_PER_PAIR * pairs,
+    }
+    names = ["sample_scan", "sample_stats", "fused_scan", "final_select", "fallback"]
+    phases = {n: statistics.mean(p[i] for p in phase_ms) for i, n in enumerate(names)}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "fp8_e4m3" if fp8 else inp.dtype, "data": "synthetic",
+        "config": {"workload": args.workload, "T": inp.T, "N": inp.N, "H": inp.H, "D": inp.D, "topk": inp.topk,
+                   "causal_offset": inp.causal_offset, "valid_pairs": pairs, "parallelism": f"replicas x{world}",
+                   "l2": "flushed between timed iterations (256 MiB write)", "workspace_bytes": int(ws.numel())},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_ms / e2e_steps},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+        "phases_ms": phases,
+        "tensor_tflops_whole_step": flops / (ms_per_step * 1e-3) / 1e12,
+        "status": {"bits": status[0], "fallback_rows": status[1], "max_survivors_per_row": status[2],
+                   "mean_survivors_per_row": status[3] / inp.T, "overflow_rows": status[4]},
+    }
+
+    if not args.no_unfused:
+        # in-repo unfused GPU baseline: dense scores to HBM in row sub-chunks, then a full-row radix select
+        buf = torch.empty(256 + (args.unfused_budget_mb << 20), dtype=torch.uint8, device="cuda")
+
+        def unfused():
+            lt.lt_unfused_topk(inp.dtype, q, w, k, ks, inp.topk, inp.causal_offset, out_idx, out_score, buf)
+
+        unfused()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        n_unf = 2
+        for _ in range(n_unf):
+            unfused()
+        e1.record(stream)
+        e1.synchronize()
+        ums = e0.elapsed_time(e1) / n_unf
+        line["unfused_gpu_baseline"] = {"value": pairs / (ums * 1e-3), "unit": UNIT, "ms_per_step": ums,
+                                        "score_buffer_mb": args.unfused_budget_mb}
+        del buf
+
+    if not args.no_cpu_baseline and world == 1:
+        v, rows, npairs, dt = time_oracle(inp, budget_s=args.cpu_budget)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                                "sample": f"{rows} evenly spaced rows x all visible keys ({npairs} pairs, {dt:.1f} s)"}
+    else:
+        line["cpu_baseline"] = None
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

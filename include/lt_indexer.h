@@ -144,6 +144,20 @@ int lt_unfused_topk(int dtype, const void* q, const float* w, const void* k, con
  */
 int lt_read_status(const void* workspace, int* status8_host, void* stream);
 
+/*
+ * Instrumentation (no counterpart in the paper; used by the benchmark).
+ *   lt_launch_count     kernels this library has launched so far in this process.
+ *   lt_set_profiling    when enabled, lt_indexer_topk(_ex) on the fused path records CUDA events on
+ *                       the caller's stream between its phases (events are created on the first
+ *                       enable for the current device).
+ *   lt_read_phase_ms    synchronises `stream` and returns the device time in ms of the five phases
+ *                       of the last profiled call: [0] sample scoring, [1] sample statistics,
+ *                       [2] fused scan (score + filter), [3] final select, [4] exact fallback.
+ */
+unsigned long long lt_launch_count(void);
+int lt_set_profiling(int enable);
+int lt_read_phase_ms(float* ms5_host, void* stream);
+
 const char* lt_strerror(int code);
 int lt_last_cuda_error(void); /* the cudaError_t behind the last LT_ERR_CUDA of this thread */
 int lt_version(void);

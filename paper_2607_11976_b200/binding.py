@@ -67,6 +67,11 @@ def load() -> ctypes.CDLL:
     lib.lt_unfused_topk.restype = i
     lib.lt_read_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int), vp]
     lib.lt_read_status.restype = i
+    lib.lt_launch_count.restype = ctypes.c_ulonglong
+    lib.lt_set_profiling.argtypes = [i]
+    lib.lt_set_profiling.restype = i
+    lib.lt_read_phase_ms.argtypes = [ctypes.POINTER(ctypes.c_float), vp]
+    lib.lt_read_phase_ms.restype = i
     lib.lt_strerror.argtypes = [i]
     lib.lt_strerror.restype = ctypes.c_char_p
     lib.lt_last_cuda_error.restype = i
@@ -153,6 +158,21 @@ def lt_read_status(workspace=None, stream=None) -> list:
     (None: the library-owned workspace of lt_indexer_topk)."""
     buf = (ctypes.c_int * 8)()
     _check(load().lt_read_status(_ptr(workspace), buf, _stream(stream)), "lt_read_status")
+    return list(buf)
+
+
+def lt_launch_count() -> int:
+    return int(load().lt_launch_count())
+
+
+def lt_set_profiling(enable: bool) -> None:
+    _check(load().lt_set_profiling(1 if enable else 0), "lt_set_profiling")
+
+
+def lt_read_phase_ms(stream=None) -> list:
+    """Device ms of [sample scoring, sample statistics, fused scan, final select, fallback]."""
+    buf = (ctypes.c_float * 5)()
+    _check(load().lt_read_phase_ms(buf, _stream(stream)), "lt_read_phase_ms")
     return list(buf)
 
 

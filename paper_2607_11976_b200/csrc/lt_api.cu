@@ -5,6 +5,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "../../include/lt_indexer.h"
@@ -16,6 +17,17 @@ namespace {
 
 thread_local int g_last_cuda_error = 0;
 
+// ---- instrumentation: kernel-launch counter and optional per-phase CUDA events ---------------
+std::atomic<unsigned long long> g_launches{0};
+constexpr int kPhases = 5;  // sample scan, sample statistics, fused scan, final select, fallback
+bool g_profiling = false;
+cudaEvent_t g_events[kPhases + 1] = {nullptr};
+int g_events_dev = -1;
+
+void mark_phase(int i, cudaStream_t stream) {
+  if (g_profiling && g_events[i] != nullptr) cudaEventRecord(g_events[i], stream);
+}
+
 #define LT_CUDA(expr)                                  \
   do {                                                 \
     cudaError_t e__ = (expr);                          \
@@ -23,6 +35,12 @@ thread_local int g_last_cuda_error = 0;
       g_last_cuda_error = static_cast<int>(e__);       \
       return LT_ERR_CUDA;                              \
     }                                                  \
+  } while (0)
+
+#define LT_LAUNCH(expr) \
+  do {                  \
+    LT_CUDA(expr);      \
+    ++g_launches;       \
   } while (0)
 
 constexpr size_t kAlign = 256;
@@ -172,9 +190,9 @@ int run_unfused(int dtype, bool mma, const void* q, const float* w, const void* 
       p.dump = scores;
       p.dump_ld = N;
       p.ctl = ctl;
-      LT_CUDA(launch_scan_mma(dtype, kModeDump, q, T, k, N, D, p, grid, stream));
+      LT_LAUNCH(launch_scan_mma(dtype, kModeDump, q, T, k, N, D, p, grid, stream));
     } else {
-      LT_CUDA(launch_simt_scores(dtype, q, w, k, k_scale, T, N, H, D, causal_offset, r0, r1, scores, N, stream));
+      LT_LAUNCH(launch_simt_scores(dtype, q, w, k, k_scale, T, N, H, D, causal_offset, r0, r1, scores, N, stream));
     }
     if (topk > 0) {
       SelectRowsParams sp{};
@@ -189,7 +207,7 @@ int run_unfused(int dtype, bool mma, const void* q, const float* w, const void* 
       sp.out_idx = out_idx;
       sp.out_score = out_score;
       sp.ctl = ctl;
-      LT_CUDA(launch_select_rows(sp, stream));
+      LT_LAUNCH(launch_select_rows(sp, stream));
     }
   }
   return LT_OK;
@@ -230,6 +248,7 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
   float* scratch = reinterpret_cast<float*>(ws + L.scratch);
 
   // 1. sample phase: score n_sample strided keys of the common prefix with the same tensor-core path
+  mark_phase(0, stream);
   if (L.n_sample > 0) {
     ScanParams p{};
     p.w = w;
@@ -246,9 +265,11 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
     p.dump = sample;
     p.dump_ld = L.n_sample;
     p.ctl = ctl;
-    LT_CUDA(launch_scan_mma(dtype, kModeDump, q, T, k, L.n_sample, static_cast<long long>(L.sample_stride) * D, p, grid, stream));
+    LT_LAUNCH(launch_scan_mma(dtype, kModeDump, q, T, k, L.n_sample, static_cast<long long>(L.sample_stride) * D, p, grid, stream));
   }
-  LT_CUDA(launch_sample_stats(sample, T, L.n_sample, topk, smin, width, thr, stream));
+  mark_phase(1, stream);
+  LT_LAUNCH(launch_sample_stats(sample, T, L.n_sample, topk, smin, width, thr, stream));
+  mark_phase(2, stream);
 
   // 2. fused scan: score, gate, compact, count
   {
@@ -272,10 +293,11 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
     p.cand = cand;
     p.cap = L.cap;
     p.ctl = ctl;
-    LT_CUDA(launch_scan_mma(dtype, kModeFilter, q, T, k, N, D, p, grid, stream));
+    LT_LAUNCH(launch_scan_mma(dtype, kModeFilter, q, T, k, N, D, p, grid, stream));
   }
 
   // 3. final select over the survivors; rows it cannot finish exactly are flagged
+  mark_phase(3, stream);
   {
     FinalSelectParams p{};
     p.tail = tail;
@@ -294,11 +316,12 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
     p.block_flag = block_flag;
     p.fb_list = fb_list;
     p.ctl = ctl;
-    LT_CUDA(launch_final_select(p, stream));
+    LT_LAUNCH(launch_final_select(p, stream));
   }
 
   // 4. exact fallback for flagged rows.  The host does not know how many there are, so it
   // enqueues enough rounds for all blocks; rounds with nothing to do exit at once.
+  mark_phase(4, stream);
   const int rounds = (L.n_blocks + L.fb_slots - 1) / L.fb_slots;
   for (int r = 0; r < rounds; ++r) {
     ScanParams p{};
@@ -320,7 +343,7 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
     p.fb_round_base = r * L.fb_slots;
     p.fb_slots = L.fb_slots;
     p.ctl = ctl;
-    LT_CUDA(launch_scan_mma(dtype, kModeDump, q, T, k, N, D, p, grid, stream));
+    LT_LAUNCH(launch_scan_mma(dtype, kModeDump, q, T, k, N, D, p, grid, stream));
     SelectRowsParams sp{};
     sp.scores = scratch;
     sp.ld = N;
@@ -336,8 +359,9 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
     sp.fb_round_base = r * L.fb_slots;
     sp.row_flag = row_flag;
     sp.ctl = ctl;
-    LT_CUDA(launch_select_rows(sp, stream));
+    LT_LAUNCH(launch_select_rows(sp, stream));
   }
+  mark_phase(5, stream);
   return LT_OK;
 }
 
@@ -444,9 +468,9 @@ int lt_indexer_scores(int dtype, const void* q, const float* w, const void* k, c
     p.dump = out_scores;
     p.dump_ld = N;
     p.ctl = ctl;
-    LT_CUDA(launch_scan_mma(dtype, kModeDump, q, T, k, N, D, p, grid, stream));
+    LT_LAUNCH(launch_scan_mma(dtype, kModeDump, q, T, k, N, D, p, grid, stream));
   } else {
-    LT_CUDA(launch_simt_scores(dtype, q, w, k, kk, T, N, H, D, causal_offset, row_begin, row_end, out_scores, N, stream));
+    LT_LAUNCH(launch_simt_scores(dtype, q, w, k, kk, T, N, H, D, causal_offset, row_begin, row_end, out_scores, N, stream));
   }
   return LT_OK;
 }
@@ -485,6 +509,33 @@ int lt_read_status(const void* workspace, int* status8_host, void* stream) {
   if (src == nullptr) return LT_ERR_WORKSPACE;
   LT_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
   LT_CUDA(cudaMemcpy(status8_host, src, 8 * sizeof(int), cudaMemcpyDeviceToHost));
+  return LT_OK;
+}
+
+unsigned long long lt_launch_count(void) { return g_launches.load(); }
+
+int lt_set_profiling(int enable) {
+  if (enable) {
+    int dev = 0;
+    LT_CUDA(cudaGetDevice(&dev));
+    if (g_events_dev != dev) {
+      for (int i = 0; i <= kPhases; ++i) {
+        if (g_events[i] != nullptr) cudaEventDestroy(g_events[i]);
+        g_events[i] = nullptr;
+        LT_CUDA(cudaEventCreate(&g_events[i]));
+      }
+      g_events_dev = dev;
+    }
+  }
+  g_profiling = enable != 0;
+  return LT_OK;
+}
+
+int lt_read_phase_ms(float* ms5_host, void* stream) {
+  if (ms5_host == nullptr) return LT_ERR_INVALID_ARG;
+  if (g_events_dev < 0) return LT_ERR_INVALID_ARG;
+  LT_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+  for (int i = 0; i < kPhases; ++i) LT_CUDA(cudaEventElapsedTime(&ms5_host[i], g_events[i], g_events[i + 1]));
   return LT_OK;
 }
 
