@@ -176,6 +176,7 @@ def main():
     ap.add_argument("--workload", default="fp8_1m")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of CPU work for the oracle baseline")
+    ap.add_argument("--rows", type=int, default=0, help="profiling aid: shrink the chunk to this many query rows")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-unfused", action="store_true")
     ap.add_argument("--unfused-budget-mb", type=int, default=2048, help="score-matrix budget of the unfused GPU baseline")
@@ -208,7 +209,7 @@ def main():
         dist.barrier()
     lt.load()
 
-    inp = make_config(args.workload)
+    inp = make_config(args.workload, T=args.rows) if args.rows else make_config(args.workload)
     pairs = inp.valid_pairs()
     flops = 2.0 * inp.H * inp.D * pairs
     q, w, k, ks = lt.to_device(inp)
@@ -227,14 +228,13 @@ def main():
         torch.cuda.synchronize()
 
     lt.lt_set_profiling(True)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
     for _ in range(args.warmup):
         step()
     status = lt.lt_read_status(ws)
     if status[0] & lt.LT_STATUS_TIMEOUT:
         raise SystemExit("device-side wait timed out; results invalid")
-
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     barrier()
     launches0 = lt.lt_launch_count()
     step_ms, phase_ms = [], []

@@ -2,20 +2,25 @@
 //
 // One CTA keeps a block of 8 query rows (8 x 64 heads = 512 operand rows of D = 128) resident in
 // shared memory and streams 128-key tiles of K past it.  Per key tile it issues two 128 x 256 x 128
-// UMMAs (4 queries each) into a two-stage ring of TMEM accumulators; lanes index keys and columns
-// index (query, head), so each epilogue thread owns one key and finishes Eq. 1 of the paper
-// (ReLU, head-weighted sum, key scale) as an in-thread FFMA chain over TMEM columns.
+// UMMAs (unit u = queries 4u .. 4u+3) into the two 256-column halves of TMEM; lanes index keys and
+// columns index (query, head), so each epilogue thread owns one key and finishes Eq. 1 of the paper
+// (ReLU, head-weighted sum, key scale) as an in-thread chain of packed FMAs over TMEM columns.
 //
 //   kMode == kModeFilter  paper Sec. 3.2 "Filtering": gate the score against the row's threshold
-//                         edge, ballot-compact the survivors of each warp into the row's candidate
-//                         buffer (one tail atomic per ballot) and count them in the row's bin
-//                         histogram; a spare warp re-derives the threshold bin from the histogram
-//                         while the scan runs ("Threshold Refresh") and publishes it by plain store.
+//                         edge, ballot-compact the survivors of each warp into a staging list and
+//                         count them in the row's bin histogram; a spare warp re-derives the
+//                         threshold bin from the histogram while the scan runs ("Threshold
+//                         Refresh") and publishes it by plain store.
 //   kMode == kModeDump    write every score (or -inf where masked) to a dense matrix: used for the
 //                         sample phase, lt_indexer_scores, the unfused baseline and the exact fallback.
 //
-// Warp roles (384 threads): 0 TMA producer, 1 UMMA issuer (+ TMEM owner), 2 threshold refresh,
-// 3 idle, 4..11 epilogue (two warpgroups; warpgroup g finishes queries 2g, 2g+1 of each unit).
+// Warp roles (608 threads): 0 TMA producer, 1 UMMA issuer (+ TMEM owner), 2 threshold refresh,
+// 3..18 epilogue in four warpgroups.  Warpgroup g finishes query g of unit 0 (TMEM half 0) and then
+// query g of unit 1 (half 1) of every key tile, so the UMMA warp refills one half while the other
+// is drained.  Inside a warp the next 32-column TMEM load (also the first one of the next half) is
+// always in flight while the previous 32 columns are reduced.  Survivors of the gate go to small
+// per-warp staging lists in shared memory and are flushed to the row's candidate buffer in batches
+// (one tail atomic per flush; paper Sec. 3.2 "Filtering").
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <math.h>
@@ -35,14 +40,17 @@ constexpr int kH = 64;
 constexpr int kD = 128;
 constexpr int kBlockQ = 8;                  // query rows resident per CTA
 constexpr int kUnitQ = 4;                   // query rows per UMMA (N = 4 * 64 = 256 columns)
-constexpr int kUnits = kBlockQ / kUnitQ;    // UMMAs per key tile
+constexpr int kUnits = kBlockQ / kUnitQ;    // UMMAs per key tile = TMEM halves
 constexpr int kUmmaN = kUnitQ * kH;         // 256
-constexpr int kTmemCols = 512;              // two accumulator stages of 256 fp32 columns
-constexpr int kEpiWarps = 8;
+constexpr int kTmemCols = 512;              // two accumulators of 256 fp32 columns
+constexpr int kFirstEpiWarp = 3;
+constexpr int kEpiWarps = 16;
 constexpr int kEpiThreads = kEpiWarps * 32;
-constexpr int kThreads = 128 + kEpiThreads;
+constexpr int kThreads = kFirstEpiWarp * 32 + kEpiThreads;
 constexpr int kSwizzleTile = 128 * 128;     // bytes: 128 rows x 128-byte swizzled rows
 constexpr int kQTile = 256 * 128;           // bytes: 256 rows x 128-byte rows (one unit, one K-half)
+constexpr int kStageLen = 64;               // entries of one per-warp staging list
+constexpr int kUnitWBytes = kUnitQ * kH * 4;  // bytes between the weights of query g and query 4 + g
 
 template <bool kFp8>
 struct Cfg {
@@ -72,6 +80,7 @@ struct SmemTail {
   int abort_flag;
   int epi_abort;
   int done_seq;
+  uint2 stage[kEpiWarps][kUnits][kStageLen];  // per warp and unit: (score bits, key index) of survivors
 };
 
 template <bool kFp8>
@@ -111,17 +120,91 @@ __device__ __forceinline__ bool resolve_item(const ScanParams& p, int n_blocks, 
   return it.tile_lo < it.tile_hi;
 }
 
-// Eq. 1 for one key against one query: 64 TMEM columns (per-head dots) -> ReLU -> weighted sum.
-// This one function produces every score the library ranks or dumps on the tensor-core path.
-__device__ __forceinline__ void head_sum32(const uint32_t (&v)[32], const float* __restrict__ w, float& acc0, float& acc1) {
-#pragma unroll
-  for (int j = 0; j < 32; j += 4) {
-    float4 ww = *reinterpret_cast<const float4*>(w + j);
-    acc0 = __fmaf_rn(ww.x, fmaxf(__uint_as_float(v[j + 0]), 0.f), acc0);
-    acc1 = __fmaf_rn(ww.y, fmaxf(__uint_as_float(v[j + 1]), 0.f), acc1);
-    acc0 = __fmaf_rn(ww.z, fmaxf(__uint_as_float(v[j + 2]), 0.f), acc0);
-    acc1 = __fmaf_rn(ww.w, fmaxf(__uint_as_float(v[j + 3]), 0.f), acc1);
+// ---- Eq. 1 for one key against one query ------------------------------------------------------
+// 32 TMEM columns (per-head dots) -> ReLU -> weighted sum, accumulated into four packed fp32 pairs
+// (eight independent chains).  Head h lands in pair (h / 2) % 4, lane h % 2; combine() fixes the
+// order of the final additions.  These functions produce every score the library ranks or dumps
+// on the tensor-core path, so fused, dumped and fallback scores agree bit for bit.
+struct Acc8 {
+  uint64_t p[4];
+};
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+// acc (+)= w * ReLU(x) for two heads at once.  The ReLU is applied in place on the two registers
+// the TMEM load filled, so that they stay an aligned register pair for the packed FMA.
+//   kSat == false: ReLU(x) = max(x, 0)                                  (ALU pipe)
+//   kSat == true : ReLU(x) = sat(x * 2^-25) * 2^25, the 2^25 being folded into the weight the
+//                  caller stored for this head                          (FMA pipe)
+// The saturating form needs |x| < 2^25 and no underflow of x * 2^-25; both hold for dot products of
+// 128 e4m3 codes (|x| <= 448^2 * 128 < 2^25, non-zero |x| >= 2^-18).  Scaling by a power of two is
+// exact, so w * 2^25 * (x * 2^-25) and w * x round to the same fp32 value: the two forms give
+// bit-identical sums and are mixed only to spread the work over both pipes.
+// kFirst: the accumulator starts at w * ReLU(x) (a multiply) instead of being zero-initialised.
+template <bool kSat, bool kFirst>
+__device__ __forceinline__ void relu_fma2(uint64_t& acc, uint64_t w, uint32_t& x0, uint32_t& x1) {
+  // everything stays in the untyped 32-bit registers of the TMEM load (no typed copies)
+  if (kSat) {
+    asm("mul.sat.f32 %0, %0, 0f33000000;" : "+r"(x0));
+    asm("mul.sat.f32 %0, %0, 0f33000000;" : "+r"(x1));
+  } else {
+    asm("max.f32 %0, %0, 0f00000000;" : "+r"(x0));
+    asm("max.f32 %0, %0, 0f00000000;" : "+r"(x1));
   }
+  if (kFirst) {
+    asm("{\n.reg .b64 x;\nmov.b64 x, {%1, %2};\nmul.rn.f32x2 %0, %3, x;\n}\n" : "=l"(acc) : "r"(x0), "r"(x1), "l"(w));
+  } else {
+    asm("{\n.reg .b64 x;\nmov.b64 x, {%1, %2};\nfma.rn.f32x2 %0, %3, x, %0;\n}\n" : "+l"(acc) : "r"(x0), "r"(x1), "l"(w));
+  }
+}
+// Weight stored in shared memory for head h: heads whose ReLU takes the saturating form carry 2^25.
+template <bool kFp8>
+__device__ __forceinline__ float stored_weight(float w, int h) {
+  return (kFp8 && (h & 2)) ? w * 33554432.f : w;
+}
+// Eight heads starting at column J of a 32-column piece.  kOff: byte offset of the piece's weights
+// from w_addr, folded into the load instructions as an immediate.
+template <bool kFp8, bool kFirst, int kOff, int J>
+__device__ __forceinline__ void head_sum8(uint32_t (&v)[32], uint32_t w_addr, Acc8& acc) {
+  uint64_t w01, w23, w45, w67;
+  asm volatile("ld.shared.v2.b64 {%0, %1}, [%2+%3];" : "=l"(w01), "=l"(w23) : "r"(w_addr), "n"(kOff + J * 4));
+  asm volatile("ld.shared.v2.b64 {%0, %1}, [%2+%3];" : "=l"(w45), "=l"(w67) : "r"(w_addr), "n"(kOff + J * 4 + 16));
+  constexpr bool first = kFirst && J == 0;
+  relu_fma2<false, first>(acc.p[0], w01, v[J + 0], v[J + 1]);
+  relu_fma2<kFp8, first>(acc.p[1], w23, v[J + 2], v[J + 3]);
+  relu_fma2<false, first>(acc.p[2], w45, v[J + 4], v[J + 5]);
+  relu_fma2<kFp8, first>(acc.p[3], w67, v[J + 6], v[J + 7]);
+}
+template <bool kFp8, bool kFirst, int kOff>
+__device__ __forceinline__ void head_sum32(uint32_t (&v)[32], uint32_t w_addr, Acc8& acc) {
+  head_sum8<kFp8, kFirst, kOff, 0>(v, w_addr, acc);
+  head_sum8<kFp8, kFirst, kOff, 8>(v, w_addr, acc);
+  head_sum8<kFp8, kFirst, kOff, 16>(v, w_addr, acc);
+  head_sum8<kFp8, kFirst, kOff, 24>(v, w_addr, acc);
+}
+__device__ __forceinline__ float combine(const Acc8& acc, float ks) {
+  uint64_t ab, cd, all;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(ab) : "l"(acc.p[0]), "l"(acc.p[1]));
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(cd) : "l"(acc.p[2]), "l"(acc.p[3]));
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(all) : "l"(ab), "l"(cd));
+  float lo, hi;
+  unpack2(all, lo, hi);
+  return __fmaf_rn(lo + hi, ks, 0.f);  // the + 0 turns -0 into +0
+}
+
+// Flush one staging list: reserve room in the row's candidate buffer with a single atomic and copy
+// the entries out with all lanes.  Entries beyond the capacity are dropped; the tail counter still
+// counts them, which is how the final select learns that the row overflowed.
+__device__ __forceinline__ void flush_stage(const uint2* list, int count, const ScanParams& p, int t, int lane) {
+  __syncwarp();
+  uint32_t base = 0;
+  if (lane == 0) base = atomicAdd(p.tail + t, static_cast<uint32_t>(count));
+  base = __shfl_sync(0xffffffffu, base, 0);
+  for (int i = lane; i < count; i += 32) {
+    uint32_t pos = base + i;
+    if (pos < static_cast<uint32_t>(p.cap)) p.cand[static_cast<size_t>(t) * p.cap + pos] = list[i];
+  }
+  __syncwarp();
 }
 
 template <bool kFp8, int kMode>
@@ -193,7 +276,7 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         Item it;
         if (!resolve_item(p, n_blocks, item, it)) continue;
         // query block: wait until the UMMAs of the previous item no longer read it
-        ok = mbar_wait(smem_u32(&st->bar_q_empty), (n_done & 1) ^ 1, abort_flag);
+        ok = mbar_wait<40>(smem_u32(&st->bar_q_empty), (n_done & 1) ^ 1, abort_flag);
         if (!ok) break;
         mbar_arrive_expect_tx(smem_u32(&st->bar_q_full), C::kQBytes);
         for (int u = 0; u < kUnits; ++u)
@@ -202,7 +285,7 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
                         (it.t0 + u * kUnitQ) * kH, smem_u32(&st->bar_q_full));
         ++n_done;
         for (int tile = it.tile_lo; tile < it.tile_hi; ++tile) {
-          ok = mbar_wait(smem_u32(&st->bar_empty[stage]), phase ^ 1, abort_flag);
+          ok = mbar_wait<40>(smem_u32(&st->bar_empty[stage]), phase ^ 1, abort_flag);
           if (!ok) break;
           mbar_arrive_expect_tx(smem_u32(&st->bar_full[stage]), C::kStageBytes);
           for (int hf = 0; hf < C::kHalves; ++hf)
@@ -221,21 +304,20 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       constexpr uint32_t idesc = make_idesc(kFp8, kUmmaN);
       int stage = 0;
       uint32_t phase = 0;
-      int acc = 0;
-      uint32_t acc_phase = 0;
+      uint32_t acc_phase = 0;  // flips once per key tile: each TMEM half is filled once per tile
       uint32_t n_done = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
         Item it;
         if (!resolve_item(p, n_blocks, item, it)) continue;
-        ok = mbar_wait(smem_u32(&st->bar_q_full), n_done & 1, abort_flag);
+        ok = mbar_wait<40>(smem_u32(&st->bar_q_full), n_done & 1, abort_flag);
         if (!ok) break;
         ++n_done;
         for (int tile = it.tile_lo; tile < it.tile_hi && ok; ++tile) {
-          ok = mbar_wait(smem_u32(&st->bar_full[stage]), phase, abort_flag);
+          ok = mbar_wait<40>(smem_u32(&st->bar_full[stage]), phase, abort_flag);
           if (!ok) break;
           for (int u = 0; u < kUnits; ++u) {
-            ok = mbar_wait(smem_u32(&st->bar_tmem_empty[acc]), acc_phase ^ 1, abort_flag);
+            ok = mbar_wait<40>(smem_u32(&st->bar_tmem_empty[u]), acc_phase ^ 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
 #pragma unroll
@@ -244,12 +326,11 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
               const int step = kFp8 ? kb : (kb & 3);
               uint64_t a = make_smem_desc_sw128(k_base + stage * C::kStageBytes + hf * kSwizzleTile) + (step * 32 >> 4);
               uint64_t b = make_smem_desc_sw128(q_base + (u * C::kHalves + hf) * kQTile) + (step * 32 >> 4);
-              tc_mma<kFp8>(tmem_base + acc * kUmmaN, a, b, idesc, kb > 0 ? 1u : 0u);
+              tc_mma<kFp8>(tmem_base + u * kUmmaN, a, b, idesc, kb > 0 ? 1u : 0u);
             }
-            tc_commit(smem_u32(&st->bar_tmem_full[acc]));
-            acc ^= 1;
-            if (acc == 0) acc_phase ^= 1;
+            tc_commit(smem_u32(&st->bar_tmem_full[u]));
           }
+          acc_phase ^= 1;
           tc_commit(smem_u32(&st->bar_empty[stage]));
           if (++stage == C::kStages) {
             stage = 0;
@@ -259,16 +340,18 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         tc_commit(smem_u32(&st->bar_q_empty));
       }
     }
-  } else if (warp == 2 || warp >= 4) {
+  } else {
     // ------------------------------------------------------------------ epilogue (+ refresh warp)
     const bool is_refresh = (warp == 2);
     const int n_sync = (kMode == kModeFilter) ? kEpiThreads + 32 : kEpiThreads;
     if (!(is_refresh && kMode != kModeFilter)) {
-      const int e = threadIdx.x - 128;        // epilogue thread number (valid for warp >= 4)
-      const int quarter = warp & 3;           // TMEM lane quarter this warp may read
-      const int g = (warp - 4) >> 2;          // warpgroup: queries 2g, 2g+1 of each unit
+      const int e = threadIdx.x - kFirstEpiWarp * 32;  // epilogue thread number (valid for epilogue warps)
+      const int ew = warp - kFirstEpiWarp;             // epilogue warp number
+      const int quarter = warp & 3;                    // TMEM lane quarter this warp may read
+      const int g = ew >> 2;                           // warpgroup 0..3: queries g (unit 0) and 4 + g (unit 1)
       const int key_in_tile = quarter * 32 + lane;
-      int acc = 0;
+      const uint32_t tcol = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(g * kH);
+      const uint32_t w_addr = smem_u32(st->w) + g * kH * 4;
       uint32_t acc_phase = 0;
       int seq = 0;
       for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
@@ -279,7 +362,7 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         if (!is_refresh) {
           for (int i = e; i < kBlockQ * kH; i += kEpiThreads) {
             int t = it.t0 + i / kH;
-            st->w[i] = (t < p.T) ? p.w[static_cast<size_t>(t) * kH + (i % kH)] : 0.f;
+            st->w[i] = (t < p.T) ? stored_weight<kFp8>(p.w[static_cast<size_t>(t) * kH + (i % kH)], i % kH) : 0.f;
           }
           if (e < kBlockQ) {
             int t = it.t0 + e;
@@ -300,9 +383,13 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         if (is_refresh) {
           // ---- paper Sec. 3.2 "Threshold Refresh": walk each row's histogram from the top bin
           // down until the cumulative count reaches k; publish the bin's lower edge by plain store.
+          // The gate moves fast only while few keys have been seen, so the polling interval grows
+          // geometrically (1 us -> 32 us): a stale edge merely admits a few more candidates, while a
+          // busy polling warp would take issue slots from the epilogue warps of its scheduler.
           int cur_tb[kBlockQ];
 #pragma unroll
           for (int r = 0; r < kBlockQ; ++r) cur_tb[r] = 0;
+          unsigned int sleep_ns = 1000;
           while (true) {
 #pragma unroll
             for (int r = 0; r < kBlockQ; ++r) {
@@ -349,77 +436,96 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
                 }
               }
             }
-            if (*reinterpret_cast<volatile int*>(&st->done_seq) >= seq || *abort_flag) break;
-            __nanosleep(400);
+            // sleep in slices so that the end of the item is noticed quickly
+            bool done = false;
+            for (unsigned int slept = 0; slept < sleep_ns && !done; slept += 1000) {
+              __nanosleep(1000);
+              done = *reinterpret_cast<volatile int*>(&st->done_seq) >= seq || *abort_flag;
+            }
+            if (done) break;
+            if (sleep_ns < 32000) sleep_ns += sleep_ns >> 1;
           }
           continue;
         }
 
-        // ---- epilogue proper
-        for (int tile = it.tile_lo; tile < it.tile_hi; ++tile) {
+        // ---- epilogue proper: this warp finishes queries g and 4 + g for its 32 keys of every tile
+        int cnt[kUnits] = {0, 0};  // entries in this warp's staging lists (warp-uniform)
+        const int vis_first = st->vis[0];
+        uint32_t va[32], vb[32];
+        // TMEM loads are issued unconditionally (a load after a failed wait only fetches values
+        // nobody uses): a conditional load would keep the previous contents of the 32 destination
+        // registers alive and cost a register copy per element.
+        bool ok = mbar_wait(smem_u32(&st->bar_tmem_full[0]), acc_phase, abort_flag);
+        tc_fence_after();
+        tmem_ld32(tcol, va);
+        for (int tile = it.tile_lo; tile < it.tile_hi && ok; ++tile) {
           const int s = tile * kTileKeys + key_in_tile;
           float ks = 1.f;
           if (p.k_scale != nullptr && s < p.n_keys) ks = __ldg(p.k_scale + static_cast<size_t>(s) * p.ks_stride);
-          bool ok = true;
+          // keys of this tile that some row of the block may not see (diagonal or ragged last tile)
+          const bool partial = (tile + 1) * kTileKeys > vis_first;
+#pragma unroll
           for (int u = 0; u < kUnits; ++u) {
-            ok = mbar_wait(smem_u32(&st->bar_tmem_full[acc]), acc_phase, abort_flag);
-            if (!ok) break;
-            tc_fence_after();
-            float score[2];
-#pragma unroll
-            for (int qq = 0; qq < 2; ++qq) {
-              const int r = u * kUnitQ + g * 2 + qq;
-              const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
-                                     static_cast<uint32_t>(acc * kUmmaN + (g * 2 + qq) * kH);
-              float acc0 = 0.f, acc1 = 0.f;
-              uint32_t v[32];
-              tmem_ld32(taddr, v);
-              tmem_ld_wait();
-              head_sum32(v, st->w + r * kH, acc0, acc1);
-              tmem_ld32(taddr + 32, v);
-              tmem_ld_wait();
-              if (qq == 1) {
-                // both queries' columns are in registers: hand the accumulator stage back
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&st->bar_tmem_empty[acc]));
-              }
-              head_sum32(v, st->w + r * kH + 32, acc0, acc1);
-              score[qq] = (acc0 + acc1) * ks + 0.f;  // + 0 turns -0 into +0
+            const int r = u * kUnitQ + g;
+            Acc8 acc;
+            // va: first 32 heads of (tile, u), already in flight
+            tmem_ld_wait();
+            tmem_ld32(tcol + u * kUmmaN + 32, vb);
+            if (u == 0) head_sum32<kFp8, true, 0>(va, w_addr, acc); else head_sum32<kFp8, true, kUnitWBytes>(va, w_addr, acc);
+            tmem_ld_wait();
+            // this warp's columns of half u are in registers: hand the half back to the UMMA warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&st->bar_tmem_empty[u]));
+            // start the first load of the next half before reducing the rest of this one
+            if (u == 0) {
+              ok = mbar_wait(smem_u32(&st->bar_tmem_full[1]), acc_phase, abort_flag);
+              tc_fence_after();
+              tmem_ld32(tcol + kUmmaN, va);
+            } else {
+              acc_phase ^= 1;
+              if (tile + 1 < it.tile_hi) ok = mbar_wait(smem_u32(&st->bar_tmem_full[0]), acc_phase, abort_flag);
+              tc_fence_after();
+              tmem_ld32(tcol, va);  // after the item's last tile this load is a dummy
             }
-            acc ^= 1;
-            if (acc == 0) acc_phase ^= 1;
-#pragma unroll
-            for (int qq = 0; qq < 2; ++qq) {
-              const int r = u * kUnitQ + g * 2 + qq;
-              const bool visible = s < st->vis[r];
-              if (kMode == kModeDump) {
-                int dr = st->dump_row[r];
-                if (dr >= 0 && s < p.n_keys) p.dump[static_cast<size_t>(dr) * p.dump_ld + s] = visible ? score[qq] : -INFINITY;
-              } else {
-                // ---- paper Sec. 3.2 "Filtering": gate, ballot-compact, batched append, histogram
-                const float thr = *reinterpret_cast<volatile float*>(&st->thr[r]);
-                const bool pass = visible && (score[qq] >= thr);
-                const uint32_t ballot = __ballot_sync(0xffffffffu, pass);
-                if (ballot != 0) {
-                  const int t = it.t0 + r;
-                  uint32_t base = 0;
-                  if (lane == 0) base = atomicAdd(p.tail + t, static_cast<uint32_t>(__popc(ballot)));
-                  base = __shfl_sync(0xffffffffu, base, 0);
-                  if (pass) {
-                    uint32_t pos = base + __popc(ballot & ((1u << lane) - 1u));
-                    if (pos < static_cast<uint32_t>(p.cap))
-                      p.cand[static_cast<size_t>(t) * p.cap + pos] = make_uint2(__float_as_uint(score[qq]), static_cast<uint32_t>(s));
-                    int b = bin_of(score[qq], st->smin[r], st->width[r]);
-                    atomicAdd(p.hist + static_cast<size_t>(t) * kBins + b, 1u);
-                  }
+            if (u == 0) head_sum32<kFp8, false, 128>(vb, w_addr, acc); else head_sum32<kFp8, false, kUnitWBytes + 128>(vb, w_addr, acc);
+            const float score = combine(acc, ks);
+            if (kMode == kModeDump) {
+              const int dr = st->dump_row[r];
+              if (dr >= 0 && s < p.n_keys)
+                p.dump[static_cast<size_t>(dr) * p.dump_ld + s] = (s < st->vis[r]) ? score : -INFINITY;
+            } else {
+              // ---- paper Sec. 3.2 "Filtering": gate, ballot-compact into the warp's staging list,
+              // count in the histogram; the list is flushed to the candidate buffer in batches
+              const float thr = *reinterpret_cast<volatile float*>(&st->thr[r]);
+              bool pass = score >= thr;
+              if (partial) pass = pass && (s < st->vis[r]);
+              const uint32_t ballot = __ballot_sync(0xffffffffu, pass);
+              if (ballot != 0) {
+                const int t = it.t0 + r;
+                const int n = __popc(ballot);
+                uint2* list = st->stage[ew][u];
+                if (cnt[u] + n > kStageLen) {
+                  flush_stage(list, cnt[u], p, t, lane);
+                  cnt[u] = 0;
                 }
+                if (pass) {
+                  list[cnt[u] + __popc(ballot & ((1u << lane) - 1u))] = make_uint2(__float_as_uint(score), static_cast<uint32_t>(s));
+                  atomicAdd(p.hist + static_cast<size_t>(t) * kBins + bin_of(score, st->smin[r], st->width[r]), 1u);
+                }
+                cnt[u] += n;
               }
             }
+            if (!ok) break;
           }
-          if (!ok) break;
         }
-        if (warp == 4 && lane == 0) *reinterpret_cast<volatile int*>(&st->done_seq) = seq;
+        tmem_ld_wait();  // the trailing load must land before its registers are reused
+        if (kMode == kModeFilter) {
+#pragma unroll
+          for (int u = 0; u < kUnits; ++u)
+            if (cnt[u] > 0) flush_stage(st->stage[ew][u], cnt[u], p, it.t0 + u * kUnitQ + g, lane);
+        }
+        if (warp == kFirstEpiWarp && lane == 0) *reinterpret_cast<volatile int*>(&st->done_seq) = seq;
       }
     }
   }
