@@ -17,8 +17,9 @@
 // Warp roles (608 threads): 0 TMA producer, 1 UMMA issuer (+ TMEM owner), 2 threshold refresh,
 // 3..18 epilogue in four warpgroups.  Warpgroup g finishes query g of unit 0 (TMEM half 0) and then
 // query g of unit 1 (half 1) of every key tile, so the UMMA warp refills one half while the other
-// is drained.  Inside a warp the next 32-column TMEM load (also the first one of the next half) is
-// always in flight while the previous 32 columns are reduced.  Survivors of the gate go to small
+// is drained.  A warp pulls its 64 columns of a half into registers with one wait, hands the half
+// back at once and only then does the arithmetic; the four warps of a scheduler cover each
+// other's barrier and TMEM latencies.  Survivors of the gate go to small
 // per-warp staging lists in shared memory and are flushed to the row's candidate buffer in batches
 // (one tail atomic per flush; paper Sec. 3.2 "Filtering").
 #include <cuda.h>
@@ -448,47 +449,54 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           continue;
         }
 
-        // ---- epilogue proper: this warp finishes queries g and 4 + g for its 32 keys of every tile
+        // ---- epilogue proper: this warp finishes queries g and 4 + g for its 32 keys of every tile.
+        // Every step with a long fixed latency is issued ahead of its use: the key scale of the
+        // next tile and the row threshold are fetched before the arithmetic of the current one.
         int cnt[kUnits] = {0, 0};  // entries in this warp's staging lists (warp-uniform)
         const int vis_first = st->vis[0];
-        uint32_t va[32], vb[32];
-        // TMEM loads are issued unconditionally (a load after a failed wait only fetches values
-        // nobody uses): a conditional load would keep the previous contents of the 32 destination
-        // registers alive and cost a register copy per element.
-        bool ok = mbar_wait(smem_u32(&st->bar_tmem_full[0]), acc_phase, abort_flag);
-        tc_fence_after();
-        tmem_ld32(tcol, va);
+        const bool has_scale = p.k_scale != nullptr;
+        bool ok = true;
+        float ks_next = 1.f;
+        {
+          const int s0 = it.tile_lo * kTileKeys + key_in_tile;
+          if (has_scale && s0 < p.n_keys) ks_next = __ldg(p.k_scale + static_cast<size_t>(s0) * p.ks_stride);
+        }
         for (int tile = it.tile_lo; tile < it.tile_hi && ok; ++tile) {
           const int s = tile * kTileKeys + key_in_tile;
-          float ks = 1.f;
-          if (p.k_scale != nullptr && s < p.n_keys) ks = __ldg(p.k_scale + static_cast<size_t>(s) * p.ks_stride);
+          const float ks = ks_next;
+          {
+            const int s1 = s + kTileKeys;
+            if (has_scale && tile + 1 < it.tile_hi && s1 < p.n_keys)
+              ks_next = __ldg(p.k_scale + static_cast<size_t>(s1) * p.ks_stride);
+          }
           // keys of this tile that some row of the block may not see (diagonal or ragged last tile)
           const bool partial = (tile + 1) * kTileKeys > vis_first;
 #pragma unroll
           for (int u = 0; u < kUnits; ++u) {
             const int r = u * kUnitQ + g;
-            Acc8 acc;
-            // va: first 32 heads of (tile, u), already in flight
-            tmem_ld_wait();
+            float thr = 0.f;
+            if (kMode == kModeFilter) thr = *reinterpret_cast<volatile float*>(&st->thr[r]);
+            ok = mbar_wait(smem_u32(&st->bar_tmem_full[u]), acc_phase, abort_flag);
+            tc_fence_after();
+            // the 64 columns of this query: both loads in flight, one wait.  The loads are issued even
+            // after a failed wait (they then fetch values nobody uses): keeping them unconditional
+            // keeps the 64 destination registers free of copies.
+            uint32_t va[32], vb[32];
+            tmem_ld32(tcol + u * kUmmaN, va);
             tmem_ld32(tcol + u * kUmmaN + 32, vb);
-            if (u == 0) head_sum32<kFp8, true, 0>(va, w_addr, acc); else head_sum32<kFp8, true, kUnitWBytes>(va, w_addr, acc);
             tmem_ld_wait();
             // this warp's columns of half u are in registers: hand the half back to the UMMA warp
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&st->bar_tmem_empty[u]));
-            // start the first load of the next half before reducing the rest of this one
+            Acc8 acc;
             if (u == 0) {
-              ok = mbar_wait(smem_u32(&st->bar_tmem_full[1]), acc_phase, abort_flag);
-              tc_fence_after();
-              tmem_ld32(tcol + kUmmaN, va);
+              head_sum32<kFp8, true, 0>(va, w_addr, acc);
+              head_sum32<kFp8, false, 128>(vb, w_addr, acc);
             } else {
-              acc_phase ^= 1;
-              if (tile + 1 < it.tile_hi) ok = mbar_wait(smem_u32(&st->bar_tmem_full[0]), acc_phase, abort_flag);
-              tc_fence_after();
-              tmem_ld32(tcol, va);  // after the item's last tile this load is a dummy
+              head_sum32<kFp8, true, kUnitWBytes>(va, w_addr, acc);
+              head_sum32<kFp8, false, kUnitWBytes + 128>(vb, w_addr, acc);
             }
-            if (u == 0) head_sum32<kFp8, false, 128>(vb, w_addr, acc); else head_sum32<kFp8, false, kUnitWBytes + 128>(vb, w_addr, acc);
             const float score = combine(acc, ks);
             if (kMode == kModeDump) {
               const int dr = st->dump_row[r];
@@ -497,7 +505,6 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             } else {
               // ---- paper Sec. 3.2 "Filtering": gate, ballot-compact into the warp's staging list,
               // count in the histogram; the list is flushed to the candidate buffer in batches
-              const float thr = *reinterpret_cast<volatile float*>(&st->thr[r]);
               bool pass = score >= thr;
               if (partial) pass = pass && (s < st->vis[r]);
               const uint32_t ballot = __ballot_sync(0xffffffffu, pass);
@@ -518,8 +525,8 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             }
             if (!ok) break;
           }
+          acc_phase ^= 1;
         }
-        tmem_ld_wait();  // the trailing load must land before its registers are reused
         if (kMode == kModeFilter) {
 #pragma unroll
           for (int u = 0; u < kUnits; ++u)
