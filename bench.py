@@ -103,6 +103,24 @@ class ClockSampler:
                 "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(value: float, world: int, device) -> float:
+    """MAX of a per-rank scalar over all ranks (the timing rule for multi-GPU numbers)."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(pairs_per_rank: int, steps: int, total_ms_max: float, world: int) -> float:
+    """Whole-job pairs/s of `world` independent replicas, each doing pairs_per_rank pairs per step,
+    when the slowest rank took total_ms_max for its steps."""
+    return world * pairs_per_rank * steps / (total_ms_max * 1e-3)
+
+
 def cpu_threads() -> int:
     try:
         from threadpoolctl import threadpool_info
@@ -250,13 +268,9 @@ def main():
     launches = lt.lt_launch_count() - launches0
     barrier()
     clocks = sampler.stop()
-    total_ms = sum(step_ms)
-    if world > 1:
-        tmax = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        total_ms = float(tmax.item())
+    total_ms = max_over_ranks(sum(step_ms), world, "cuda")
     ms_per_step = total_ms / args.steps
-    value = world * pairs * args.steps / (total_ms * 1e-3)
+    value = aggregate_throughput(pairs, args.steps, total_ms, world)
     status = lt.lt_read_status(ws)
 
     # ---- end to end through the public API with host buffers: H2D of the inputs, D2H of the result
@@ -283,12 +297,8 @@ def main():
         e2e_step()
     e1.record(stream)
     e1.synchronize()
-    e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        tmax = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tmax.item())
-    e2e_value = world * pairs * e2e_steps / (e2e_ms * 1e-3)
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
+    e2e_value = aggregate_throughput(pairs, e2e_steps, e2e_ms, world)
 
     if rank != 0:
         if world > 1:

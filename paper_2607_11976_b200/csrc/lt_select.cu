@@ -134,14 +134,20 @@ __device__ __forceinline__ void sort_and_write(uint64_t* sel, int count, int top
 }
 
 // ---------------------------------------------------------------------------------------------
-// final select over one row's candidate buffer.
+// final select over one row's candidate buffer (paper Sec. 3.2 "Top-k Selection"): the final
+// threshold bin is the highest bin whose cumulative count from the top reaches k; every candidate
+// at or above its lower edge is pulled into shared memory (the bins above hold fewer than k of
+// them), sorted by (score desc, index asc), and the first k are written out.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kSelThreads) final_select_kernel(const FinalSelectParams p) {
-  extern __shared__ uint64_t sel[];  // kSelCap keys
+constexpr int kFinalThreads = 512;
+
+__global__ void __launch_bounds__(kFinalThreads) final_select_kernel(const FinalSelectParams p, int sel_cap) {
+  extern __shared__ uint64_t sel[];  // sel_cap keys
   __shared__ unsigned int hist[kBins];
   __shared__ int s_tb;
   __shared__ unsigned int s_count;
   const int t = blockIdx.x;
+  const int lane = threadIdx.x & 31;
   const unsigned int tail = p.tail[t];
   const int vis = visible_keys(t, p.N, p.causal_offset);
   const int kk = p.topk < vis ? p.topk : vis;
@@ -155,34 +161,73 @@ __global__ void __launch_bounds__(kSelThreads) final_select_kernel(const FinalSe
     if (threadIdx.x < kBins) hist[threadIdx.x] = p.hist[static_cast<size_t>(t) * kBins + threadIdx.x];
     if (threadIdx.x == 0) s_count = 0;
     __syncthreads();
-    if (threadIdx.x == 0) {
-      // final threshold bin: the bins above it hold fewer than k candidates
+    if (threadIdx.x < 32) {
+      // suffix sums over the 256 bins, 8 bins per lane, exactly as the refresh warp of the scan does
+      unsigned int c[8];
+      unsigned int mine = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        c[j] = hist[lane * 8 + j];
+        mine += c[j];
+      }
+      unsigned int incl = mine;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        unsigned int o = __shfl_down_sync(0xffffffffu, incl, d);
+        if (lane + d < 32) incl += o;
+      }
+      const unsigned int above = incl - mine;
+      const unsigned int need = static_cast<unsigned int>(kk);
       int tb = 0;
-      unsigned int cum = 0;
-      for (int b = kBins - 1; b >= 1; --b) {
-        cum += hist[b];
-        if (cum >= static_cast<unsigned int>(kk)) {
-          tb = b;
-          break;
+      if (above < need && incl >= need) {
+        unsigned int cum = above;
+        for (int j = 7; j >= 0; --j) {
+          cum += c[j];
+          if (cum >= need) {
+            tb = lane * 8 + j;
+            break;
+          }
         }
       }
-      s_tb = tb;
+      // bin 0 is "everything else": a crossing inside lane 0 may legitimately report bin 0
+      tb = __reduce_max_sync(0xffffffffu, tb);
+      if (need == 0) tb = kBins - 1;
+      if (lane == 0) s_tb = tb;
     }
     __syncthreads();
     const float edge = bin_edge(s_tb, p.smin[t], p.width[t]);
     const uint2* cand = p.cand + static_cast<size_t>(t) * p.cap;
-    for (unsigned int i = threadIdx.x; i < tail; i += kSelThreads) {
-      uint2 c = cand[i];
-      float sc = __uint_as_float(c.x);
-      if (sc >= edge) {
-        unsigned int pos = atomicAdd(&s_count, 1u);
-        if (pos < static_cast<unsigned int>(kSelCap)) sel[pos] = pack_key(sc, static_cast<int>(c.y));
+    // candidates are fetched eight rounds at a time so that the loads of a batch overlap
+    constexpr int kBatch = 8;
+    const unsigned int rounds = (tail + kFinalThreads - 1) / kFinalThreads;
+    for (unsigned int r0 = 0; r0 < rounds; r0 += kBatch) {
+      uint2 c[kBatch];
+#pragma unroll
+      for (int j = 0; j < kBatch; ++j) {
+        const unsigned int i = (r0 + j) * kFinalThreads + threadIdx.x;
+        c[j] = (i < tail) ? __ldcs(cand + i) : make_uint2(0xff800000u, 0u);  // -inf never passes a finite edge
+      }
+#pragma unroll
+      for (int j = 0; j < kBatch; ++j) {
+        const unsigned int i = (r0 + j) * kFinalThreads + threadIdx.x;
+        const bool take = (i < tail) && (__uint_as_float(c[j].x) >= edge);
+        // one shared-memory atomic per warp
+        const unsigned int ballot = __ballot_sync(0xffffffffu, take);
+        if (ballot != 0) {
+          unsigned int base = 0;
+          if (lane == 0) base = atomicAdd(&s_count, static_cast<unsigned int>(__popc(ballot)));
+          base = __shfl_sync(0xffffffffu, base, 0);
+          if (take) {
+            const unsigned int pos = base + __popc(ballot & ((1u << lane) - 1u));
+            if (pos < static_cast<unsigned int>(sel_cap)) sel[pos] = pack_key(__uint_as_float(c[j].x), static_cast<int>(c[j].y));
+          }
+        }
       }
     }
     __syncthreads();
     const unsigned int count = s_count;
     // count < kk cannot happen for an exact filter; treating it as "redo" keeps the result exact regardless
-    if (count > static_cast<unsigned int>(kSelCap) || count < static_cast<unsigned int>(kk)) redo = true;
+    if (count > static_cast<unsigned int>(sel_cap) || count < static_cast<unsigned int>(kk)) redo = true;
     if (!redo) {
       sort_and_write(sel, static_cast<int>(count), p.topk, p.out_idx + static_cast<size_t>(t) * p.topk,
                      p.out_score ? p.out_score + static_cast<size_t>(t) * p.topk : nullptr);
@@ -341,10 +386,14 @@ cudaError_t launch_sample_stats(const float* sample, int T, int n_sample, int to
 }
 
 cudaError_t launch_final_select(const FinalSelectParams& p, cudaStream_t stream) {
-  const int smem = kSelCap * sizeof(uint64_t);
+  // room for every candidate at or above the final threshold edge: normally a little more than k
+  int sel_cap = next_pow2(4 * p.topk);
+  if (sel_cap < 2048) sel_cap = 2048;
+  if (sel_cap > kSelCap) sel_cap = kSelCap;
+  const int smem = sel_cap * static_cast<int>(sizeof(uint64_t));
   cudaError_t e = cudaFuncSetAttribute(final_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
-  final_select_kernel<<<p.T, kSelThreads, smem, stream>>>(p);
+  final_select_kernel<<<p.T, kFinalThreads, smem, stream>>>(p, sel_cap);
   return cudaGetLastError();
 }
 
