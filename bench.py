@@ -34,9 +34,11 @@ UNIT = "pairs/s"
 NOMINAL_FP8_TFLOPS = 4500.0
 NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM bytes of one launch of the fused scan kernel (dram__bytes_read.sum + dram__bytes_write.sum),
-# per scored pair, from the ncu capture summarised under profiles/; scaled by the pairs of a launch.
-SCAN_DRAM_BYTES_PER_PAIR = None
+# DRAM bytes of one launch of the fused scan kernel (dram__bytes_read.sum + dram__bytes_write.sum) from
+# the ncu capture of a 592-row case summarised in profiles/scan_kernel_fp8_T592_N1M.md: 207.2 MB, of which
+# the key stream (N * D bytes, read once whatever the number of rows) is 134.2 MB and the rest
+# (candidate write-back, queries, weights) grows with the rows: (207.2 - 134.2) MB / 592 rows.
+SCAN_TRAFFIC = {"fp8_1m": {"fixed_bytes": 134.2e6, "bytes_per_row": (207.2e6 - 134.2e6) / 592}}
 
 
 def load_peaks():
@@ -119,6 +121,13 @@ def aggregate_throughput(pairs_per_rank: int, steps: int, total_ms_max: float, w
     """Whole-job pairs/s of `world` independent replicas, each doing pairs_per_rank pairs per step,
     when the slowest rank took total_ms_max for its steps."""
     return world * pairs_per_rank * steps / (total_ms_max * 1e-3)
+
+
+def algorithmic_bytes(inp) -> int:
+    """Minimum HBM traffic of one call: read q, w, k (+ k_scale) once, write indices and scores."""
+    esz = {"f32": 4, "bf16": 2, "e4m3": 1}[inp.dtype]
+    reads = inp.T * inp.H * inp.D * esz + inp.T * inp.H * 4 + inp.N * inp.D * esz + (inp.N * 4 if inp.k_scale is not None else 0)
+    return reads + inp.T * inp.topk * 8
 
 
 def cpu_threads() -> int:
@@ -316,7 +325,9 @@ def main():
         "unit": "TFLOP/s", "frac": achieved / peak_tflops, "peak_kind": f"of {peak_kind} (bf16 burst x {2 if fp8 else 1})",
         "frac_of_nominal": achieved / (NOMINAL_FP8_TFLOPS if fp8 else NOMINAL_BF16_TFLOPS),
         "flops_per_launch": flops, "kernel_ms": scan_ms,
-        "traffic": None if SCAN_DRAM_BYTES_PER_PAIR is None else SCAN_DRAM_BYTES_PER_PAIR * pairs,
+        "traffic": (SCAN_TRAFFIC[args.workload]["fixed_bytes"] + SCAN_TRAFFIC[args.workload]["bytes_per_row"] * inp.T)
+        if args.workload in SCAN_TRAFFIC else None,
+        "algorithmic_bytes": algorithmic_bytes(inp),
     }
     names = ["sample_scan", "sample_stats", "fused_scan", "final_select", "fallback"]
     phases = {n: statistics.mean(p[i] for p in phase_ms) for i, n in enumerate(names)}
