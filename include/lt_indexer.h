@@ -61,6 +61,7 @@ extern "C" {
 #define LT_ERR_UNSUPPORTED (-2) /* dtype / shape the library has no path for                              */
 #define LT_ERR_WORKSPACE (-3)   /* workspace missing, misaligned or too small                             */
 #define LT_ERR_CUDA (-4)        /* a CUDA runtime call failed; see lt_last_cuda_error                     */
+#define LT_ERR_TOO_LARGE (-5)   /* lt_indexer_topk_static: the problem does not fit the fixed scratch     */
 
 /* bits of the device status word (lt_read_status, status[0]) */
 #define LT_STATUS_TIMEOUT 1  /* a bounded device-side wait ran out; results are invalid   */
@@ -134,6 +135,41 @@ int lt_unfused_topk(int dtype, const void* q, const float* w, const void* k, con
                     int T, int N, int H, int D, int topk, int causal_offset,
                     int32_t* out_idx, float* out_score,
                     float* score_buf, size_t score_buf_bytes, int path, void* stream);
+
+/*
+ * Exact indexer top-k for callers that must not allocate device memory.  (The paper has no
+ * counterpart: this entry point exists for deployment reasons only.)
+ *
+ * Who needs it: a serving process that hands nearly all free HBM to its KV cache at start-up (the
+ * paper's Sec. 1 budget leaves under 3 GB of headroom) cannot count on a later cudaMalloc to
+ * succeed, and a caller in a latency-critical loop cannot afford the device-wide synchronisation a
+ * cudaMalloc or cudaFree implies.  Such callers also often have no workspace of their own to lend.
+ *
+ * What it does: the same result as lt_indexer_topk_ex (same outputs, same ordering, same scores bit
+ * for bit), computed by the decoupled path - dense scores of a few rows at a time, then a full-row
+ * radix select - whose scratch is a fixed LT_STATIC_SCRATCH_BYTES array inside the library's device
+ * image instead of a caller workspace.  Every GPU that loads the library holds that array until the
+ * process exits.  The call itself performs no cudaMalloc, cudaFree or other allocating call; q, w,
+ * k, k_scale, out_idx, out_score are the caller's device buffers as everywhere else.
+ *
+ * Limits and rules:
+ *   - one score row must fit: N * 4 <= LT_STATIC_SCRATCH_BYTES - 256 (N <= 4,194,240), otherwise
+ *     LT_ERR_TOO_LARGE is returned and nothing is enqueued; rows are processed
+ *     floor((LT_STATIC_SCRATCH_BYTES - 256) / (4 N)) at a time, so large T x N problems run as many
+ *     small passes and are slower than lt_indexer_topk_ex;
+ *   - the first call on each device looks up the array's device address (cudaGetSymbolAddress);
+ *     make that first call before any stream capture begins on that device;
+ *   - all calls on a device share the one array, which keeps the previous call's contents (the call
+ *     clears the status block it needs at zero and overwrites score rows before reading them):
+ *     two calls whose kernels may overlap on the GPU (different streams, or different host threads
+ *     on different streams) race on it - serialise them on one stream;
+ *   - the status block is not readable through lt_read_status; device-side waits are bounded as in
+ *     every other entry point.
+ */
+#define LT_STATIC_SCRATCH_BYTES (16u << 20)
+int lt_indexer_topk_static(int dtype, const void* q, const float* w, const void* k, const float* k_scale,
+                           int T, int N, int H, int D, int topk, int causal_offset,
+                           int32_t* out_idx, float* out_score, void* stream);
 
 /*
  * Copies the 8-int status block of a workspace to host memory after synchronising

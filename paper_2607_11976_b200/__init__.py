@@ -16,6 +16,7 @@ from .binding import (  # noqa: F401
     lt_indexer_scores,
     lt_indexer_topk,
     lt_indexer_topk_ex,
+    lt_indexer_topk_static,
     lt_indexer_topk_workspace_bytes,
     lt_read_status,
     lt_unfused_topk,

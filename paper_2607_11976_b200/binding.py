@@ -65,6 +65,8 @@ def load() -> ctypes.CDLL:
     lib.lt_indexer_scores.restype = i
     lib.lt_unfused_topk.argtypes = [i, vp, fp, vp, fp, i, i, i, i, i, i, ip, fp, fp, sz, i, vp]
     lib.lt_unfused_topk.restype = i
+    lib.lt_indexer_topk_static.argtypes = [i, vp, fp, vp, fp, i, i, i, i, i, i, ip, fp, vp]
+    lib.lt_indexer_topk_static.restype = i
     lib.lt_read_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int), vp]
     lib.lt_read_status.restype = i
     lib.lt_launch_count.restype = ctypes.c_ulonglong
@@ -151,6 +153,15 @@ def lt_unfused_topk(dtype, q, w, k, k_scale, topk: int, causal_offset: int, out_
     _check(load().lt_unfused_topk(dtype_code(dtype), _ptr(q), _ptr(w), _ptr(k), _ptr(k_scale), T, N, H, D, topk,
                                   causal_offset, _ptr(out_idx), _ptr(out_score), _ptr(score_buf),
                                   score_buf.numel() * score_buf.element_size(), path, _stream(stream)), "lt_unfused_topk")
+
+
+def lt_indexer_topk_static(dtype, q, w, k, k_scale, topk: int, causal_offset: int, out_idx, out_score=None, stream=None) -> None:
+    """Allocation-free entry point: same result as lt_indexer_topk_ex, scratch inside the library
+    (16 MiB per GPU, one score row must fit: N <= 4,194,240).  Calls that may overlap on the GPU race."""
+    T, N, H, D = _shape(q, k)
+    _check(load().lt_indexer_topk_static(dtype_code(dtype), _ptr(q), _ptr(w), _ptr(k), _ptr(k_scale), T, N, H, D, topk,
+                                         causal_offset, _ptr(out_idx), _ptr(out_score), _stream(stream)),
+           "lt_indexer_topk_static")
 
 
 def lt_read_status(workspace=None, stream=None) -> list:

@@ -365,6 +365,31 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
   return LT_OK;
 }
 
+// ---- fixed scratch of the allocation-free entry point -------------------------------------------
+// Lives in the library's device image: every GPU whose context loads the library holds these
+// 16 MiB until the process exits.  Layout: a 256-byte status block, then dense fp32 score rows.
+constexpr size_t kStaticScratchBytes = LT_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// In host code `g_static_scratch` is only a handle for the runtime, not a device address; the
+// address each device gave the array is looked up once per device and cached here.
+std::mutex g_static_mu;
+void* g_static_ptr[64] = {nullptr};
+
+int static_scratch_address(void** out) {
+  int dev = 0;
+  LT_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return LT_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  if (g_static_ptr[dev] == nullptr) {
+    void* ptr = nullptr;
+    LT_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
+    g_static_ptr[dev] = ptr;
+  }
+  *out = g_static_ptr[dev];
+  return LT_OK;
+}
+
 // ---- library-owned workspace of the 13-argument entry point -----------------------------------
 std::mutex g_arena_mu;
 void* g_arena = nullptr;
@@ -387,6 +412,7 @@ const char* lt_strerror(int code) {
     case LT_ERR_UNSUPPORTED: return "unsupported dtype or shape";
     case LT_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case LT_ERR_CUDA: return "CUDA runtime error";
+    case LT_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of lt_indexer_topk_static (N * 4 bytes must fit in LT_STATIC_SCRATCH_BYTES - 256)";
     default: return "unknown error code";
   }
 }
@@ -495,6 +521,31 @@ int lt_unfused_topk(int dtype, const void* q, const float* w, const void* k, con
   Control* ctl = reinterpret_cast<Control*>(score_buf);
   LT_CUDA(cudaMemsetAsync(ctl, 0, kAlign, stream));
   float* scores = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(score_buf) + kAlign);
+  return run_unfused(dtype, mma, q, w, k, k_scale, T, N, H, D, topk, causal_offset, out_idx, out_score, scores,
+                     static_cast<int>(rows), ctl, tun, stream);
+}
+
+int lt_indexer_topk_static(int dtype, const void* q, const float* w, const void* k, const float* k_scale, int T, int N, int H,
+                           int D, int topk, int causal_offset, int32_t* out_idx, float* out_score, void* stream_) {
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  int rc = check_problem(dtype, q, w, k, k_scale, T, N, H, D);
+  if (rc != LT_OK) return rc;
+  if (out_idx == nullptr || topk <= 0 || topk > N || topk > LT_MAX_TOPK) return LT_ERR_INVALID_ARG;
+  // one dense score row (N floats) must fit behind the status block
+  if (static_cast<size_t>(N) * 4 > kStaticScratchBytes - kAlign) return LT_ERR_TOO_LARGE;
+  void* base = nullptr;
+  rc = static_scratch_address(&base);  // the first call on a device looks the address up
+  if (rc != LT_OK) return rc;
+  Tun tun = resolve_tunables(nullptr);
+  const bool mma = use_fused(tun, dtype, H, D);
+  long long rows = static_cast<long long>((kStaticScratchBytes - kAlign) / (static_cast<size_t>(N) * 4));
+  if (rows > T) rows = T;
+  if (mma && rows >= kRowsPerBlock) rows -= rows % kRowsPerBlock;
+  // the array keeps whatever the previous call left: the status block must start at zero; the
+  // score rows are fully rewritten before they are read
+  Control* ctl = static_cast<Control*>(base);
+  LT_CUDA(cudaMemsetAsync(ctl, 0, kAlign, stream));
+  float* scores = reinterpret_cast<float*>(static_cast<unsigned char*>(base) + kAlign);
   return run_unfused(dtype, mma, q, w, k, k_scale, T, N, H, D, topk, causal_offset, out_idx, out_score, scores,
                      static_cast<int>(rows), ctl, tun, stream);
 }
