@@ -117,6 +117,20 @@ def test_no_masking_single_row_and_topk_equals_n():
     assert sorted(idx[0].tolist()) == list(range(300))
 
 
+def test_largest_topk_and_single_row_long_context():
+    # topk at the library maximum (8192) on both the fused and the generic path
+    inp = make_inputs("iid", "bf16", T=10, N=40000, H=64, D=128, topk=8192, seed=31)
+    idx, score, status = run_topk(inp, lt.Tunables(path=lt.LT_PATH_FUSED))
+    assert status[0] & lt.LT_STATUS_TIMEOUT == 0
+    assert_matches_oracle(inp, idx, score, list(range(inp.T)), dump_scores(inp, 0, inp.T, lt.LT_PATH_FUSED))
+    g_idx, g_score, _ = run_topk(inp, lt.Tunables(path=lt.LT_PATH_GENERIC))
+    assert_matches_oracle(inp, g_idx, g_score, list(range(inp.T)), dump_scores(inp, 0, inp.T, lt.LT_PATH_GENERIC))
+    # one decode-like row against a long context (many key segments, a single query block)
+    one = make_inputs("ar1", "e4m3", T=1, N=300000, H=64, D=128, topk=2048, seed=32)
+    idx, score, _ = run_topk(one, lt.Tunables(path=lt.LT_PATH_FUSED))
+    assert_matches_oracle(one, idx, score, [0], dump_scores(one, 0, 1, lt.LT_PATH_FUSED))
+
+
 def test_rows_that_see_nothing():
     inp = make_inputs("iid", "bf16", T=16, N=500, H=64, D=128, topk=8, seed=12, causal_offset=-5)
     idx, score, _ = run_topk(inp, lt.Tunables(path=lt.LT_PATH_FUSED))
