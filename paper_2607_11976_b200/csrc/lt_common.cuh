@@ -53,14 +53,19 @@ __device__ __forceinline__ float key_score(uint64_t key) {
 __device__ __forceinline__ float bin_edge(int b, float smin, float width) {
   return b <= 0 ? -INFINITY : __fmaf_rn(static_cast<float>(b), width, smin);
 }
-__device__ __forceinline__ int bin_of(float s, float smin, float width) {
+// `inv_width` is only used for a first guess (1 / width, any rounding); the edge comparisons that
+// follow decide, so the result does not depend on it.
+__device__ __forceinline__ int bin_of(float s, float smin, float width, float inv_width) {
   if (!(s >= bin_edge(1, smin, width))) return 0;
   if (!(width > 0.f)) return kBins - 1;  // degenerate range: every edge equals s_min
-  float g = (s - smin) / width;
+  float g = (s - smin) * inv_width;
   int b = g >= static_cast<float>(kBins - 1) ? kBins - 1 : (g < 1.f ? 1 : static_cast<int>(g));
   while (b < kBins - 1 && s >= bin_edge(b + 1, smin, width)) ++b;
   while (b > 1 && s < bin_edge(b, smin, width)) --b;
   return b;
+}
+__device__ __forceinline__ int bin_of(float s, float smin, float width) {
+  return bin_of(s, smin, width, width > 0.f ? 1.f / width : 0.f);
 }
 
 // ---------------------------------------------------------------------------------------------

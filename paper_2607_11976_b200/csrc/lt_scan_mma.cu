@@ -7,8 +7,9 @@
 // (ReLU, head-weighted sum, key scale) as an in-thread chain of packed FMAs over TMEM columns.
 //
 //   kMode == kModeFilter  paper Sec. 3.2 "Filtering": gate the score against the row's threshold
-//                         edge, ballot-compact the survivors of each warp into a staging list and
-//                         count them in the row's bin histogram; a spare warp re-derives the
+//                         edge, ballot-compact the survivors of each warp into a staging list; a flush
+//                         appends the list to the row's candidate buffer and counts its entries in the
+//                         row's bin histogram; a spare warp re-derives the
 //                         threshold bin from the histogram while the scan runs ("Threshold
 //                         Refresh") and publishes it by plain store.
 //   kMode == kModeDump    write every score (or -inf where masked) to a dense matrix: used for the
@@ -69,6 +70,7 @@ struct SmemTail {
   float thr[kBlockQ];
   float smin[kBlockQ];
   float width[kBlockQ];
+  float inv_width[kBlockQ];
   int vis[kBlockQ];
   int dump_row[kBlockQ];
   uint64_t bar_full[8];
@@ -193,17 +195,25 @@ __device__ __forceinline__ float combine(const Acc8& acc, float ks) {
   return __fmaf_rn(lo + hi, ks, 0.f);  // the + 0 turns -0 into +0
 }
 
-// Flush one staging list: reserve room in the row's candidate buffer with a single atomic and copy
-// the entries out with all lanes.  Entries beyond the capacity are dropped; the tail counter still
-// counts them, which is how the final select learns that the row overflowed.
-__device__ __forceinline__ void flush_stage(const uint2* list, int count, const ScanParams& p, int t, int lane) {
+// Flush one staging list: reserve room in the row's candidate buffer with a single atomic, copy the
+// entries out with all lanes and count each of them in the row's histogram (fire-and-forget
+// atomics).  Doing the bin arithmetic here, 32 entries at a time, keeps it out of the per-tile path;
+// the refresh warp merely sees the counts a little later, which can only leave the gate looser.
+// Entries beyond the capacity are dropped but still counted, and the tail counter runs past the
+// capacity, which is how the final select learns that the row overflowed.
+__device__ __forceinline__ void flush_stage(const uint2* list, int count, const ScanParams& p, int t, int lane, float smin,
+                                            float width, float inv_width) {
   __syncwarp();
   uint32_t base = 0;
   if (lane == 0) base = atomicAdd(p.tail + t, static_cast<uint32_t>(count));
   base = __shfl_sync(0xffffffffu, base, 0);
+  unsigned int* hist = p.hist + static_cast<size_t>(t) * kBins;
+  uint2* cand = p.cand + static_cast<size_t>(t) * p.cap;
   for (int i = lane; i < count; i += 32) {
-    uint32_t pos = base + i;
-    if (pos < static_cast<uint32_t>(p.cap)) p.cand[static_cast<size_t>(t) * p.cap + pos] = list[i];
+    const uint2 e = list[i];
+    const uint32_t pos = base + i;
+    if (pos < static_cast<uint32_t>(p.cap)) cand[pos] = e;
+    atomicAdd(hist + bin_of(__uint_as_float(e.x), smin, width, inv_width), 1u);
   }
   __syncwarp();
 }
@@ -374,6 +384,7 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
               st->thr[e] = live ? __ldcg(p.thr + t) : INFINITY;
               st->smin[e] = live ? p.smin[t] : 0.f;
               st->width[e] = live ? p.width[t] : 0.f;
+              st->inv_width[e] = (live && p.width[t] > 0.f) ? 1.f / p.width[t] : 0.f;
             }
           }
           if (e == 0) st->epi_abort = *abort_flag;
@@ -513,13 +524,10 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
                 const int n = __popc(ballot);
                 uint2* list = st->stage[ew][u];
                 if (cnt[u] + n > kStageLen) {
-                  flush_stage(list, cnt[u], p, t, lane);
+                  flush_stage(list, cnt[u], p, t, lane, st->smin[r], st->width[r], st->inv_width[r]);
                   cnt[u] = 0;
                 }
-                if (pass) {
-                  list[cnt[u] + __popc(ballot & ((1u << lane) - 1u))] = make_uint2(__float_as_uint(score), static_cast<uint32_t>(s));
-                  atomicAdd(p.hist + static_cast<size_t>(t) * kBins + bin_of(score, st->smin[r], st->width[r]), 1u);
-                }
+                if (pass) list[cnt[u] + __popc(ballot & ((1u << lane) - 1u))] = make_uint2(__float_as_uint(score), static_cast<uint32_t>(s));
                 cnt[u] += n;
               }
             }
@@ -530,7 +538,10 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         if (kMode == kModeFilter) {
 #pragma unroll
           for (int u = 0; u < kUnits; ++u)
-            if (cnt[u] > 0) flush_stage(st->stage[ew][u], cnt[u], p, it.t0 + u * kUnitQ + g, lane);
+            if (cnt[u] > 0) {
+              const int r = u * kUnitQ + g;
+              flush_stage(st->stage[ew][u], cnt[u], p, it.t0 + r, lane, st->smin[r], st->width[r], st->inv_width[r]);
+            }
         }
         if (warp == kFirstEpiWarp && lane == 0) *reinterpret_cast<volatile int*>(&st->done_seq) = seq;
       }
