@@ -87,7 +87,15 @@ typedef struct lt_tunables {
   int sample_mult;   /* sample size k' = sample_mult * topk (default 3, paper Sec. 3.2)  */
   int segment_tiles; /* key tiles (128 keys each) per work item (default 256)            */
   int grid;          /* CTAs of the scan kernel (default: number of SMs)                 */
-  int reserved[3];
+  int sample_rank;   /* initial gate = lower edge of the bin holding the sample's r-th largest
+                        score.  0 (default): r = ceil(m + 5 sqrt(m) + 5) capped at topk, where
+                        m = topk * k' / (keys the sample is drawn from) is the expected number of
+                        sampled keys inside the true top-k; the sample then misjudges a row with
+                        probability < 1e-6 (Poisson tail), and such a row is caught by the final
+                        select (fewer than topk survivors) and redone by the exact fallback.
+                        -1: r = topk, the paper's rule (Sec. 3.2 "Sampling"), which can never
+                        misjudge but starts ~k'/r times looser.  > 0: r itself.              */
+  int reserved[2];
 } lt_tunables;
 
 /*
@@ -114,6 +122,15 @@ int lt_indexer_topk_ex(int dtype, const void* q, const float* w, const void* k, 
 /* Bytes of workspace lt_indexer_topk_ex needs for this problem (0 on invalid arguments). */
 size_t lt_indexer_topk_workspace_bytes(int dtype, int T, int N, int H, int D, int topk,
                                        const lt_tunables* tunables);
+
+/*
+ * Host-only helper (no GPU work): the sample plan the fused path would use for this problem.
+ * plan3[0] = sample size k', plan3[1] = stride between sampled key positions (the sample is
+ * positions 0, stride, 2 stride, ... of the keys every row of the chunk can see), plan3[2] = rank r
+ * of the sampled score whose bin sets the initial gate (see lt_tunables.sample_rank).
+ * Returns LT_OK or LT_ERR_INVALID_ARG.
+ */
+int lt_indexer_sample_plan(int N, int topk, int causal_offset, const lt_tunables* tunables, int plan3[3]);
 
 /*
  * Dense scores of rows [row_begin, row_end) (Eq. 1), for debugging and parity:

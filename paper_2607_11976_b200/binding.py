@@ -34,7 +34,8 @@ class Tunables(ctypes.Structure):
     """Mirror of `lt_tunables`; zero fields mean "default"."""
 
     _fields_ = [("path", ctypes.c_int), ("cap_mult", ctypes.c_int), ("sample_mult", ctypes.c_int),
-                ("segment_tiles", ctypes.c_int), ("grid", ctypes.c_int), ("reserved", ctypes.c_int * 3)]
+                ("segment_tiles", ctypes.c_int), ("grid", ctypes.c_int), ("sample_rank", ctypes.c_int),
+                ("reserved", ctypes.c_int * 2)]
 
 
 _lib = None
@@ -61,6 +62,8 @@ def load() -> ctypes.CDLL:
     lib.lt_indexer_topk_ex.restype = i
     lib.lt_indexer_topk_workspace_bytes.argtypes = [i, i, i, i, i, i, ctypes.POINTER(Tunables)]
     lib.lt_indexer_topk_workspace_bytes.restype = sz
+    lib.lt_indexer_sample_plan.argtypes = [i, i, i, ctypes.POINTER(Tunables), ctypes.POINTER(ctypes.c_int)]
+    lib.lt_indexer_sample_plan.restype = i
     lib.lt_indexer_scores.argtypes = [i, vp, fp, vp, fp, i, i, i, i, i, i, i, fp, i, vp]
     lib.lt_indexer_scores.restype = i
     lib.lt_unfused_topk.argtypes = [i, vp, fp, vp, fp, i, i, i, i, i, i, ip, fp, fp, sz, i, vp]
@@ -122,6 +125,14 @@ def lt_indexer_topk_workspace_bytes(dtype, T: int, N: int, H: int, D: int, topk:
                                     tunables: Optional[Tunables] = None) -> int:
     return int(load().lt_indexer_topk_workspace_bytes(dtype_code(dtype), T, N, H, D, topk,
                                                       ctypes.byref(tunables) if tunables else None))
+
+
+def lt_indexer_sample_plan(N: int, topk: int, causal_offset: int, tunables: Optional[Tunables] = None):
+    """(sample size, stride, rank) the fused path uses for this problem; host-only."""
+    buf = (ctypes.c_int * 3)()
+    _check(load().lt_indexer_sample_plan(N, topk, causal_offset, ctypes.byref(tunables) if tunables else None, buf),
+           "lt_indexer_sample_plan")
+    return tuple(buf)
 
 
 def lt_indexer_topk(q, w, k, k_scale, topk: int, causal_offset: int, out_idx, out_score=None, stream=None) -> None:

@@ -1,6 +1,7 @@
 // C ABI of the indexer top-k library: argument checks, workspace layout, kernel sequencing.
 #include <cuda_runtime.h>
 #include <limits.h>
+#include <math.h>
 #include <stdint.h>
 #include <stdio.h>
 #include <string.h>
@@ -50,16 +51,17 @@ constexpr size_t kFallbackScratchBudget = size_t(512) << 20;  // dense scores ke
 constexpr size_t kGenericScratchBudget = size_t(256) << 20;   // dense scores kept at once by the generic path
 
 struct Tun {
-  int path, cap_mult, sample_mult, segment_tiles, grid;
+  int path, cap_mult, sample_mult, segment_tiles, grid, sample_rank;
 };
 Tun resolve_tunables(const lt_tunables* t) {
-  Tun r{LT_PATH_AUTO, 12, 3, 0, 0};
+  Tun r{LT_PATH_AUTO, 12, 3, 0, 0, 0};
   if (t != nullptr) {
     r.path = t->path;
     if (t->cap_mult > 0) r.cap_mult = t->cap_mult;
     if (t->sample_mult > 0) r.sample_mult = t->sample_mult;
     if (t->segment_tiles > 0) r.segment_tiles = t->segment_tiles;
     if (t->grid > 0) r.grid = t->grid;
+    r.sample_rank = t->sample_rank;
   }
   return r;
 }
@@ -86,7 +88,7 @@ struct Layout {
   // zeroed region
   size_t ctl, tail, hist, row_flag, block_flag, zero_end;
   size_t smin, width, thr, fb_list, sample, cand, scratch, total;
-  int cap, n_sample, sample_stride, fb_slots, n_blocks, generic_rows;
+  int cap, n_sample, sample_stride, sample_rank, fb_slots, n_blocks, generic_rows;
 };
 
 Layout make_layout(bool fused, int T, int N, int topk, int causal_offset, const Tun& tun) {
@@ -129,6 +131,19 @@ Layout make_layout(bool fused, int T, int N, int topk, int causal_offset, const 
   long long want = static_cast<long long>(tun.sample_mult) * topk;
   L.n_sample = static_cast<int>(want < prefix ? want : prefix);
   L.sample_stride = L.n_sample > 0 ? static_cast<int>(prefix / L.n_sample) : 1;
+  // Rank of the sampled score that sets the initial gate.  A row's true top-k holds about
+  // m = topk * n_sample / prefix sampled keys (fewer for rows that see keys past the prefix); the gate
+  // is too tight only if it holds at least `rank` of them, so rank = m + 5 sqrt(m) + 5 keeps that below
+  // 1e-6 per row (Poisson tail), and the final select sends such a row to the exact fallback.
+  if (tun.sample_rank > 0) {
+    L.sample_rank = tun.sample_rank < topk ? tun.sample_rank : topk;
+  } else if (tun.sample_rank < 0 || L.n_sample <= 0) {
+    L.sample_rank = topk;
+  } else {
+    const double m = static_cast<double>(topk) * L.n_sample / static_cast<double>(prefix);
+    const double r = ceil(m + 5.0 * sqrt(m) + 5.0);
+    L.sample_rank = r < static_cast<double>(topk) ? static_cast<int>(r) : topk;
+  }
   L.sample = off;
   off = align_up(off + static_cast<size_t>(T) * (L.n_sample > 0 ? L.n_sample : 1) * 4);
   long long cap = static_cast<long long>(tun.cap_mult) * topk;
@@ -268,7 +283,7 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
     LT_LAUNCH(launch_scan_mma(dtype, kModeDump, q, T, k, L.n_sample, static_cast<long long>(L.sample_stride) * D, p, grid, stream));
   }
   mark_phase(1, stream);
-  LT_LAUNCH(launch_sample_stats(sample, T, L.n_sample, topk, smin, width, thr, stream));
+  LT_LAUNCH(launch_sample_stats(sample, T, L.n_sample, L.sample_rank, smin, width, thr, stream));
   mark_phase(2, stream);
 
   // 2. fused scan: score, gate, compact, count
@@ -426,6 +441,15 @@ size_t lt_indexer_topk_workspace_bytes(int dtype, int T, int N, int H, int D, in
   const Tun tun = resolve_tunables(tunables);
   // the sample can never be larger with a different causal_offset than with the whole context visible
   return make_layout(use_fused(tun, dtype, H, D), T, N, topk, N - 1, tun).total;
+}
+
+int lt_indexer_sample_plan(int N, int topk, int causal_offset, const lt_tunables* tunables, int plan3[3]) {
+  if (plan3 == nullptr || N <= 0 || topk <= 0 || topk > N || topk > LT_MAX_TOPK) return LT_ERR_INVALID_ARG;
+  const Layout L = make_layout(true, 1, N, topk, causal_offset, resolve_tunables(tunables));
+  plan3[0] = L.n_sample;
+  plan3[1] = L.sample_stride;
+  plan3[2] = L.sample_rank;
+  return LT_OK;
 }
 
 int lt_indexer_topk_ex(int dtype, const void* q, const float* w, const void* k, const float* k_scale, int T, int N, int H, int D,

@@ -58,8 +58,8 @@ cudaError_t launch_simt_scores(int dtype, const void* q, const float* w, const v
                                cudaStream_t stream);
 
 // Sample statistics (paper Sec. 3.2 "Sampling"): per row min / max of the sampled scores, bin
-// width, and the threshold edge of the bin holding the k-th largest sampled score.
-cudaError_t launch_sample_stats(const float* sample, int T, int n_sample, int topk, float* smin, float* width, float* thr,
+// width, and the threshold edge of the bin holding the rank-th largest sampled score.
+cudaError_t launch_sample_stats(const float* sample, int T, int n_sample, int rank, float* smin, float* width, float* thr,
                                 cudaStream_t stream);
 
 // Final selection from the candidate buffers (paper Sec. 3.2 "Top-k Selection"); rows that cannot

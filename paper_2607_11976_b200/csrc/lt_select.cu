@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(128) simt_scores_kernel(const void* __restrict
 // ---------------------------------------------------------------------------------------------
 // sample statistics: one CTA per row.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) sample_stats_kernel(const float* __restrict__ sample, int n_sample, int topk,
+__global__ void __launch_bounds__(256) sample_stats_kernel(const float* __restrict__ sample, int n_sample, int rank,
                                                            float* __restrict__ smin_out, float* __restrict__ width_out,
                                                            float* __restrict__ thr_out) {
   __shared__ float red_min[8], red_max[8];
@@ -102,12 +102,12 @@ __global__ void __launch_bounds__(256) sample_stats_kernel(const float* __restri
   for (int i = threadIdx.x; i < n_sample; i += 256) atomicAdd(&hist[bin_of(row[i], smin, width)], 1u);
   __syncthreads();
   if (threadIdx.x == 0) {
-    // threshold bin = bin holding the k-th largest sampled score; 0 (accept all) if the sample is smaller than k
+    // threshold bin = bin holding the rank-th largest sampled score; 0 (accept all) if the sample is smaller than that
     int tb = 0;
     unsigned int cum = 0;
     for (int b = kBins - 1; b >= 1; --b) {
       cum += hist[b];
-      if (cum >= static_cast<unsigned int>(topk)) {
+      if (cum >= static_cast<unsigned int>(rank)) {
         tb = b;
         break;
       }
@@ -379,9 +379,9 @@ cudaError_t launch_simt_scores(int dtype, const void* q, const float* w, const v
   return cudaGetLastError();
 }
 
-cudaError_t launch_sample_stats(const float* sample, int T, int n_sample, int topk, float* smin, float* width, float* thr,
+cudaError_t launch_sample_stats(const float* sample, int T, int n_sample, int rank, float* smin, float* width, float* thr,
                                 cudaStream_t stream) {
-  sample_stats_kernel<<<T, 256, 0, stream>>>(sample, n_sample, topk, smin, width, thr);
+  sample_stats_kernel<<<T, 256, 0, stream>>>(sample, n_sample, rank, smin, width, thr);
   return cudaGetLastError();
 }
 

@@ -80,3 +80,29 @@ def test_workspace_arithmetic(lib):
     # generic path: a bounded dense-score scratch
     g = binding.lt_indexer_topk_workspace_bytes("f32", 64, 4096, 8, 64, 256)
     assert 64 * 4096 * 4 <= g <= 64 * 4096 * 4 + 4096
+
+
+def test_sample_plan_rank_keeps_misjudgement_below_1e6(lib):
+    """The initial gate is too tight for a row only if at least `rank` of the sampled keys fall inside
+    the row's true top-k.  With the sample a fixed fraction of the positions the chunk shares and the
+    top-k positions unrelated to the stride, that count is hypergeometric; its tail must stay below
+    the 1e-6 the header promises.  The paper's rule (rank = topk) can never misjudge."""
+    from scipy.stats import hypergeom
+
+    for N, topk, causal_offset in [(1048576, 2048, 1048576 - 4096), (131072, 2048, 131072 - 8192), (65536, 2048, 61440),
+                                   (65536, 64, 61440), (65536, 4096, 61440), (4096, 256, 4032), (16384, 256, 16320),
+                                   (1 << 22, 8192, (1 << 22) - 128), (20000, 256, 19960)]:
+        n_sample, stride, rank = binding.lt_indexer_sample_plan(N, topk, causal_offset)
+        prefix = min(causal_offset + 1, N)
+        assert n_sample == min(3 * topk, prefix) and stride == prefix // n_sample and 1 <= rank <= topk
+        if rank < topk:
+            # worst case for the tail: all topk of the row's best keys lie in the sampled prefix
+            tail = hypergeom.sf(rank - 1, prefix, topk, n_sample)
+            assert tail < 1e-6, (N, topk, rank, tail)
+        n2, s2, r2 = binding.lt_indexer_sample_plan(N, topk, causal_offset, binding.Tunables(sample_rank=-1))
+        assert (n2, s2, r2) == (n_sample, stride, topk)
+        assert binding.lt_indexer_sample_plan(N, topk, causal_offset, binding.Tunables(sample_rank=7))[2] == min(7, topk)
+    # a sample that is the whole prefix is exhaustive: the deterministic rank is used
+    assert binding.lt_indexer_sample_plan(4096, 2048, 4095)[2] == 2048
+    buf = (ctypes.c_int * 3)()
+    assert lib.lt_indexer_sample_plan(100, 200, 50, None, buf) == -1

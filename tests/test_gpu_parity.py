@@ -194,12 +194,25 @@ def test_forced_overflow_matches_default_bits():
     assert np.array_equal(idx, base_idx) and np.array_equal(score.view(np.uint32), base_score.view(np.uint32))
 
 
+def test_misjudging_sample_is_caught_and_redone_exactly():
+    # rank 1: the initial gate sits at the largest sampled score, far above the true k-th score, so most
+    # rows end the scan with fewer than topk survivors; the final select must flag them for the exact fallback
+    inp = make_config("fp8_ar1", T=40, N=20000, topk=256)
+    base_idx, base_score, st0 = run_topk(inp, lt.Tunables(path=lt.LT_PATH_FUSED))
+    idx, score, st = run_topk(inp, lt.Tunables(path=lt.LT_PATH_FUSED, sample_rank=1))
+    assert st0[1] == 0
+    assert st[1] > 0 and st[0] & lt.LT_STATUS_FALLBACK
+    assert np.array_equal(idx, base_idx) and np.array_equal(score.view(np.uint32), base_score.view(np.uint32))
+    assert_matches_oracle(inp, idx, score, list(range(0, inp.T, 7)))
+
+
 @pytest.mark.parametrize("name", ["dsa_bf16", "fp8_ar1"])
 def test_tunables_do_not_change_any_output_bit(name):
     inp = make_config(name, T=72, N=30000, topk=512)
     base_idx, base_score, _ = run_topk(inp, lt.Tunables(path=lt.LT_PATH_FUSED))
     for tun in (lt.Tunables(segment_tiles=3), lt.Tunables(segment_tiles=1000, grid=5), lt.Tunables(sample_mult=1),
-                lt.Tunables(sample_mult=8, cap_mult=20), lt.Tunables(grid=296, segment_tiles=16)):
+                lt.Tunables(sample_mult=8, cap_mult=20), lt.Tunables(grid=296, segment_tiles=16),
+                lt.Tunables(sample_rank=-1), lt.Tunables(sample_rank=100), lt.Tunables(sample_rank=10 ** 6)):
         tun.path = lt.LT_PATH_FUSED
         idx, score, st = run_topk(inp, tun)
         assert st[0] & lt.LT_STATUS_TIMEOUT == 0
