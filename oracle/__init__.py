@@ -11,3 +11,4 @@ from .indexer_topk import (  # noqa: F401
     select_topk,
     visible_keys,
 )
+from .sampler import frequent_positions, position_counts  # noqa: F401,E402

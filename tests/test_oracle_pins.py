@@ -322,3 +322,52 @@ def test_select_topk_signed_zero_and_padding():
     assert idx.tolist() == [1, 0, -1, -1] and np.isneginf(val[2:]).all()
     idx, _ = select_topk(np.zeros(0), 2)
     assert idx.tolist() == [-1, -1]
+
+
+# ---------------------------------------------------------------------------------------------
+# previous-chunk sampler (paper Sec. 3.2 "Sampling"): most frequent positions of a top-k matrix
+# ---------------------------------------------------------------------------------------------
+
+def test_frequent_positions_matches_counter_brute_force():
+    from collections import Counter
+
+    from oracle import frequent_positions
+
+    rng = np.random.default_rng(11)
+    for trial in range(40):
+        N = int(rng.integers(5, 60))
+        T = int(rng.integers(1, 12))
+        k = int(rng.integers(1, min(N, 9) + 1))
+        idx = np.stack([rng.permutation(N)[:k] for _ in range(T)]).astype(np.int64)
+        idx[rng.random(idx.shape) < 0.1] = -1  # padding entries
+        n_out = int(rng.integers(1, N + 1))
+        c = Counter(int(v) for v in idx.reshape(-1) if v >= 0)
+        ranked = sorted(range(N), key=lambda p: (-c.get(p, 0), p))[:n_out]
+        pos, cnt = frequent_positions(idx, N, n_out)
+        assert pos.tolist() == ranked
+        assert cnt.tolist() == [c.get(p, 0) for p in ranked]
+
+
+def test_frequent_positions_closed_form_and_invariants():
+    from oracle import frequent_positions
+
+    # position p appears in exactly (p % 7) rows -> ranking is by p % 7 descending, then p ascending
+    N, T = 50, 6
+    rows = [[p for p in range(N) if p % 7 > t] for t in range(T)]
+    width = max(len(r) for r in rows)
+    idx = np.full((T, width), -1, dtype=np.int64)
+    for t, r in enumerate(rows):
+        idx[t, :len(r)] = r
+    pos, cnt = frequent_positions(idx, N, N)
+    expect = sorted(range(N), key=lambda p: (-(p % 7), p))
+    assert pos.tolist() == expect and cnt.tolist() == [p % 7 for p in expect]
+    # invariants: distinct, counts non-increasing, a prefix of the full ranking, blind to row/slot order
+    rng = np.random.default_rng(5)
+    idx = rng.integers(0, 200, size=(30, 16))
+    pos, cnt = frequent_positions(idx, 200, 48)
+    assert len(set(pos.tolist())) == 48 and np.all(np.diff(cnt) <= 0)
+    assert cnt.sum() <= idx.size and pos.tolist() == frequent_positions(idx, 200, 200)[0][:48].tolist()
+    shuffled = rng.permuted(idx[rng.permutation(30)], axis=1)
+    assert frequent_positions(shuffled, 200, 48)[0].tolist() == pos.tolist()
+    with pytest.raises(ValueError):
+        frequent_positions(idx, 100, 10)
