@@ -204,6 +204,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of CPU work for the oracle baseline")
     ap.add_argument("--rows", type=int, default=0, help="profiling aid: shrink the chunk to this many query rows")
+    ap.add_argument("--sampler", default="strided", choices=["strided", "prev_chunk"],
+                    help="prev_chunk: the sample is the 3k most frequent top-k positions of the previous chunk "
+                         "(computed untimed through lt_topk_frequent; paper Sec. 3.2 'Sampling')")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-unfused", action="store_true")
     ap.add_argument("--unfused-budget-mb", type=int, default=2048, help="score-matrix budget of the unfused GPU baseline")
@@ -237,17 +240,54 @@ def main():
     lt.load()
 
     inp = make_config(args.workload, T=args.rows) if args.rows else make_config(args.workload)
+    sampler_info = None
+    sample_idx = None
+    if args.sampler == "prev_chunk":
+        # two consecutive chunks of one context: the first one is run once, untimed, to produce the sample
+        import dataclasses
+
+        T = inp.T
+        both = make_config(args.workload, T=2 * T)
+        n_prev = both.causal_offset + T
+        prev = dataclasses.replace(both, q=both.q[:T], w=both.w[:T], k=both.k[:n_prev],
+                                   k_scale=None if both.k_scale is None else both.k_scale[:n_prev])
+        inp = dataclasses.replace(both, q=both.q[T:], w=both.w[T:], causal_offset=both.causal_offset + T)
+        pq, pw, pk, pks = lt.to_device(prev)
+        p_idx = torch.empty((T, prev.topk), dtype=torch.int32, device="cuda")
+        p_ws = lt.alloc_workspace(prev.dtype, T, prev.N, prev.H, prev.D, prev.topk)
+        lt.lt_indexer_topk_ex(prev.dtype, pq, pw, pk, pks, prev.topk, prev.causal_offset, p_idx, None, p_ws)
+        n_sample = min(3 * prev.topk, lt.LT_MAX_TOPK, prev.N)
+        sample_idx = torch.empty(n_sample, dtype=torch.int32, device="cuda")
+        f_ws = torch.empty(lt.lt_topk_frequent_workspace_bytes(prev.N), dtype=torch.uint8, device="cuda")
+        lt.lt_topk_frequent(p_idx, prev.N, sample_idx, None, f_ws)
+        torch.cuda.synchronize()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(torch.cuda.current_stream())
+        for _ in range(5):
+            lt.lt_topk_frequent(p_idx, prev.N, sample_idx, None, f_ws)
+        f1.record(torch.cuda.current_stream())
+        f1.synchronize()
+        sampler_info = {"kind": "prev_chunk", "n_sample": n_sample, "previous_chunk_rows": T,
+                        "lt_topk_frequent_ms": f0.elapsed_time(f1) / 5, "timed_in_step": False}
+        del pq, pw, pk, pks, p_ws, f_ws
     pairs = inp.valid_pairs()
     flops = 2.0 * inp.H * inp.D * pairs
     q, w, k, ks = lt.to_device(inp)
     out_idx = torch.empty((inp.T, inp.topk), dtype=torch.int32, device="cuda")
     out_score = torch.empty((inp.T, inp.topk), dtype=torch.float32, device="cuda")
-    ws = lt.alloc_workspace(inp.dtype, inp.T, inp.N, inp.H, inp.D, inp.topk)
+    if sample_idx is None:
+        ws = lt.alloc_workspace(inp.dtype, inp.T, inp.N, inp.H, inp.D, inp.topk)
+    else:
+        ws = torch.empty(lt.lt_indexer_topk_sampled_workspace_bytes(inp.dtype, inp.T, inp.N, inp.H, inp.D, inp.topk,
+                                                                    sample_idx.numel()), dtype=torch.uint8, device="cuda")
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")  # larger than the 126 MB L2
     stream = torch.cuda.current_stream()
 
     def step():
-        lt.lt_indexer_topk_ex(inp.dtype, q, w, k, ks, inp.topk, inp.causal_offset, out_idx, out_score, ws)
+        if sample_idx is None:
+            lt.lt_indexer_topk_ex(inp.dtype, q, w, k, ks, inp.topk, inp.causal_offset, out_idx, out_score, ws)
+        else:
+            lt.lt_indexer_topk_sampled(inp.dtype, q, w, k, ks, inp.topk, inp.causal_offset, sample_idx, out_idx, out_score, ws)
 
     def barrier():
         if world > 1:
@@ -346,6 +386,7 @@ def main():
         "roofline": roofline,
         "phases_ms": phases,
         "tensor_tflops_whole_step": flops / (ms_per_step * 1e-3) / 1e12,
+        "sampler": sampler_info or {"kind": "strided"},
         "status": {"bits": status[0], "fallback_rows": status[1], "max_survivors_per_row": status[2],
                    "mean_survivors_per_row": status[3] / inp.T, "overflow_rows": status[4]},
     }

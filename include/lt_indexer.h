@@ -124,6 +124,47 @@ size_t lt_indexer_topk_workspace_bytes(int dtype, int T, int N, int H, int D, in
                                        const lt_tunables* tunables);
 
 /*
+ * Fused indexer top-k with a caller-provided sample (paper Sec. 3.2 "Sampling": for sparse attention
+ * the sample of a chunk is the k' = 3k positions most frequent in the previous chunk's top-k, see
+ * lt_topk_frequent).  Same outputs as lt_indexer_topk_ex, bit for bit, whatever the sample holds:
+ * the sample only decides how tight the initial gate is.
+ *   sample_idx  device, n_sample key positions (int32).  They should be distinct and visible to every
+ *               row of the chunk (0 <= position <= causal_offset); the initial gate is then the bin of
+ *               the topk-th largest sampled score, which can never misjudge (the sample is a subset of
+ *               every row's keys).  Positions outside [0, N) are read as position 0; duplicates,
+ *               positions past causal_offset or such replaced positions can at worst make the gate too
+ *               tight for some rows, which the final select detects and the exact fallback redoes.
+ *   n_sample    1 .. LT_MAX_SAMPLE.  Fewer than topk positions leave the gate open until the
+ *               online refresh takes over.
+ *   workspace   at least lt_indexer_topk_sampled_workspace_bytes(...) bytes.
+ * lt_tunables.sample_mult is ignored; sample_rank > 0 overrides the rank, otherwise rank = topk.
+ * On shapes the fused path does not support the sample is ignored.
+ */
+#define LT_MAX_SAMPLE 32768
+int lt_indexer_topk_sampled(int dtype, const void* q, const float* w, const void* k, const float* k_scale,
+                            int T, int N, int H, int D, int topk, int causal_offset,
+                            const int32_t* sample_idx, int n_sample,
+                            int32_t* out_idx, float* out_score,
+                            void* workspace, size_t workspace_bytes, const lt_tunables* tunables, void* stream);
+size_t lt_indexer_topk_sampled_workspace_bytes(int dtype, int T, int N, int H, int D, int topk, int n_sample,
+                                               const lt_tunables* tunables);
+
+/*
+ * The n_out positions that occur most often in a chunk's top-k index matrix (paper Sec. 3.2
+ * "Sampling": the previous-chunk sampler), ordered by (count descending, position ascending);
+ * positions that never occur (count 0) fill the tail in ascending order.
+ *   idx        device, [T][topk] int32 as written by the top-k entry points; entries < 0 are padding
+ *              and entries >= N are ignored
+ *   out_pos    device, n_out int32;  out_count: device, n_out int32, or NULL
+ *   n_out      1 .. min(N, LT_MAX_TOPK)
+ *   workspace  device, 256-byte aligned, at least lt_topk_frequent_workspace_bytes(N) bytes (about 4 N)
+ * Integer work only: the result is exact.  Enqueued on `stream`; no host synchronisation.
+ */
+int lt_topk_frequent(const int32_t* idx, int T, int topk, int N, int n_out, int32_t* out_pos, int32_t* out_count,
+                     void* workspace, size_t workspace_bytes, void* stream);
+size_t lt_topk_frequent_workspace_bytes(int N);
+
+/*
  * Host-only helper (no GPU work): the sample plan the fused path would use for this problem.
  * plan3[0] = sample size k', plan3[1] = stride between sampled key positions (the sample is
  * positions 0, stride, 2 stride, ... of the keys every row of the chunk can see), plan3[2] = rank r

@@ -62,6 +62,14 @@ def load() -> ctypes.CDLL:
     lib.lt_indexer_topk_ex.restype = i
     lib.lt_indexer_topk_workspace_bytes.argtypes = [i, i, i, i, i, i, ctypes.POINTER(Tunables)]
     lib.lt_indexer_topk_workspace_bytes.restype = sz
+    lib.lt_indexer_topk_sampled.argtypes = [i, vp, fp, vp, fp, i, i, i, i, i, i, ip, i, ip, fp, vp, sz, ctypes.POINTER(Tunables), vp]
+    lib.lt_indexer_topk_sampled.restype = i
+    lib.lt_indexer_topk_sampled_workspace_bytes.argtypes = [i, i, i, i, i, i, i, ctypes.POINTER(Tunables)]
+    lib.lt_indexer_topk_sampled_workspace_bytes.restype = sz
+    lib.lt_topk_frequent.argtypes = [ip, i, i, i, i, ip, ip, vp, sz, vp]
+    lib.lt_topk_frequent.restype = i
+    lib.lt_topk_frequent_workspace_bytes.argtypes = [i]
+    lib.lt_topk_frequent_workspace_bytes.restype = sz
     lib.lt_indexer_sample_plan.argtypes = [i, i, i, ctypes.POINTER(Tunables), ctypes.POINTER(ctypes.c_int)]
     lib.lt_indexer_sample_plan.restype = i
     lib.lt_indexer_scores.argtypes = [i, vp, fp, vp, fp, i, i, i, i, i, i, i, fp, i, vp]
@@ -149,6 +157,34 @@ def lt_indexer_topk_ex(dtype, q, w, k, k_scale, topk: int, causal_offset: int, o
                                      causal_offset, _ptr(out_idx), _ptr(out_score), _ptr(workspace),
                                      workspace.numel() * workspace.element_size(),
                                      ctypes.byref(tunables) if tunables else None, _stream(stream)), "lt_indexer_topk_ex")
+
+
+def lt_indexer_topk_sampled_workspace_bytes(dtype, T: int, N: int, H: int, D: int, topk: int, n_sample: int,
+                                            tunables: Optional[Tunables] = None) -> int:
+    return int(load().lt_indexer_topk_sampled_workspace_bytes(dtype_code(dtype), T, N, H, D, topk, n_sample,
+                                                              ctypes.byref(tunables) if tunables else None))
+
+
+def lt_indexer_topk_sampled(dtype, q, w, k, k_scale, topk: int, causal_offset: int, sample_idx, out_idx, out_score, workspace,
+                            tunables: Optional[Tunables] = None, stream=None) -> None:
+    """lt_indexer_topk_ex with a caller-provided sample (int32 device tensor of key positions)."""
+    T, N, H, D = _shape(q, k)
+    _check(load().lt_indexer_topk_sampled(dtype_code(dtype), _ptr(q), _ptr(w), _ptr(k), _ptr(k_scale), T, N, H, D, topk,
+                                          causal_offset, _ptr(sample_idx), sample_idx.numel(), _ptr(out_idx), _ptr(out_score),
+                                          _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                          ctypes.byref(tunables) if tunables else None, _stream(stream)),
+           "lt_indexer_topk_sampled")
+
+
+def lt_topk_frequent_workspace_bytes(N: int) -> int:
+    return int(load().lt_topk_frequent_workspace_bytes(N))
+
+
+def lt_topk_frequent(idx, N: int, out_pos, out_count, workspace, stream=None) -> None:
+    """out_pos (int32 device tensor of n_out elements) = the most frequent positions of the [T, topk] matrix idx."""
+    T, topk = idx.shape
+    _check(load().lt_topk_frequent(_ptr(idx), T, topk, N, out_pos.numel(), _ptr(out_pos), _ptr(out_count), _ptr(workspace),
+                                   workspace.numel() * workspace.element_size(), _stream(stream)), "lt_topk_frequent")
 
 
 def lt_indexer_scores(dtype, q, w, k, k_scale, causal_offset: int, row_begin: int, row_end: int, out_scores,

@@ -87,11 +87,14 @@ struct Layout {
   bool fused;
   // zeroed region
   size_t ctl, tail, hist, row_flag, block_flag, zero_end;
-  size_t smin, width, thr, fb_list, sample, cand, scratch, total;
+  size_t smin, width, thr, fb_list, sample, gather_k, gather_scale, cand, scratch, total;
   int cap, n_sample, sample_stride, sample_rank, fb_slots, n_blocks, generic_rows;
 };
 
-Layout make_layout(bool fused, int T, int N, int topk, int causal_offset, const Tun& tun) {
+// n_given > 0: the caller provides that many sample positions (lt_indexer_topk_sampled); their keys are
+// gathered into a dense buffer of the workspace (key_row_bytes each) and scored from there.
+Layout make_layout(bool fused, int T, int N, int topk, int causal_offset, const Tun& tun, int n_given = 0,
+                   int key_row_bytes = 0) {
   Layout L{};
   L.fused = fused;
   size_t off = 0;
@@ -131,14 +134,18 @@ Layout make_layout(bool fused, int T, int N, int topk, int causal_offset, const 
   long long want = static_cast<long long>(tun.sample_mult) * topk;
   L.n_sample = static_cast<int>(want < prefix ? want : prefix);
   L.sample_stride = L.n_sample > 0 ? static_cast<int>(prefix / L.n_sample) : 1;
+  if (n_given > 0) {
+    L.n_sample = n_given;
+    L.sample_stride = 1;
+  }
   // Rank of the sampled score that sets the initial gate.  A row's true top-k holds about
   // m = topk * n_sample / prefix sampled keys (fewer for rows that see keys past the prefix); the gate
   // is too tight only if it holds at least `rank` of them, so rank = m + 5 sqrt(m) + 5 keeps that below
   // 1e-6 per row (Poisson tail), and the final select sends such a row to the exact fallback.
   if (tun.sample_rank > 0) {
     L.sample_rank = tun.sample_rank < topk ? tun.sample_rank : topk;
-  } else if (tun.sample_rank < 0 || L.n_sample <= 0) {
-    L.sample_rank = topk;
+  } else if (tun.sample_rank < 0 || L.n_sample <= 0 || n_given > 0) {
+    L.sample_rank = topk;  // the paper's rule; a caller-provided sample is not a uniform one
   } else {
     const double m = static_cast<double>(topk) * L.n_sample / static_cast<double>(prefix);
     const double r = ceil(m + 5.0 * sqrt(m) + 5.0);
@@ -146,6 +153,10 @@ Layout make_layout(bool fused, int T, int N, int topk, int causal_offset, const 
   }
   L.sample = off;
   off = align_up(off + static_cast<size_t>(T) * (L.n_sample > 0 ? L.n_sample : 1) * 4);
+  L.gather_k = off;
+  off = align_up(off + static_cast<size_t>(n_given) * key_row_bytes);
+  L.gather_scale = off;
+  off = align_up(off + static_cast<size_t>(n_given) * 4);
   long long cap = static_cast<long long>(tun.cap_mult) * topk;
   L.cap = static_cast<int>(cap > N ? N : cap);
   L.cand = off;
@@ -228,16 +239,19 @@ int run_unfused(int dtype, bool mma, const void* q, const float* w, const void* 
   return LT_OK;
 }
 
+size_t elem_bytes(int dtype) { return dtype == LT_DTYPE_F32 ? 4 : (dtype == LT_DTYPE_BF16 ? 2 : 1); }
+
 int topk_impl(int dtype, const void* q, const float* w, const void* k, const float* k_scale, int T, int N, int H, int D, int topk,
               int causal_offset, int32_t* out_idx, float* out_score, void* workspace, size_t workspace_bytes,
-              const lt_tunables* tunables, cudaStream_t stream) {
+              const lt_tunables* tunables, cudaStream_t stream, const int32_t* sample_idx = nullptr, int n_given = 0) {
   int rc = check_problem(dtype, q, w, k, k_scale, T, N, H, D);
   if (rc != LT_OK) return rc;
   if (out_idx == nullptr || topk <= 0 || topk > N || topk > LT_MAX_TOPK) return LT_ERR_INVALID_ARG;
   const Tun tun = resolve_tunables(tunables);
   const bool fused = use_fused(tun, dtype, H, D);
   if (tun.path == LT_PATH_FUSED && !fused) return LT_ERR_UNSUPPORTED;
-  const Layout L = make_layout(fused, T, N, topk, causal_offset, tun);
+  const int key_row_bytes = static_cast<int>(static_cast<size_t>(D) * elem_bytes(dtype));
+  const Layout L = make_layout(fused, T, N, topk, causal_offset, tun, n_given, key_row_bytes);
   if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) != 0 || workspace_bytes < L.total)
     return LT_ERR_WORKSPACE;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
@@ -263,11 +277,20 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
   float* scratch = reinterpret_cast<float*>(ws + L.scratch);
 
   // 1. sample phase: score n_sample strided keys of the common prefix with the same tensor-core path
+  //    (or, with a caller-provided sample, a dense copy of the keys at the given positions)
   mark_phase(0, stream);
+  const void* sample_keys = k;
+  const float* sample_scale = k_scale;
+  if (n_given > 0) {
+    LT_LAUNCH(launch_gather_keys(k, k_scale, sample_idx, n_given, N, key_row_bytes, ws + L.gather_k,
+                                 reinterpret_cast<float*>(ws + L.gather_scale), stream));
+    sample_keys = ws + L.gather_k;
+    if (k_scale != nullptr) sample_scale = reinterpret_cast<const float*>(ws + L.gather_scale);
+  }
   if (L.n_sample > 0) {
     ScanParams p{};
     p.w = w;
-    p.k_scale = k_scale;
+    p.k_scale = sample_scale;
     p.ks_stride = L.sample_stride;
     p.T = T;
     p.row_begin = 0;
@@ -280,7 +303,8 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
     p.dump = sample;
     p.dump_ld = L.n_sample;
     p.ctl = ctl;
-    LT_LAUNCH(launch_scan_mma(dtype, kModeDump, q, T, k, L.n_sample, static_cast<long long>(L.sample_stride) * D, p, grid, stream));
+    LT_LAUNCH(launch_scan_mma(dtype, kModeDump, q, T, sample_keys, L.n_sample, static_cast<long long>(L.sample_stride) * D, p, grid,
+                              stream));
   }
   mark_phase(1, stream);
   LT_LAUNCH(launch_sample_stats(sample, T, L.n_sample, L.sample_rank, smin, width, thr, stream));
@@ -441,6 +465,64 @@ size_t lt_indexer_topk_workspace_bytes(int dtype, int T, int N, int H, int D, in
   const Tun tun = resolve_tunables(tunables);
   // the sample can never be larger with a different causal_offset than with the whole context visible
   return make_layout(use_fused(tun, dtype, H, D), T, N, topk, N - 1, tun).total;
+}
+
+int lt_indexer_topk_sampled(int dtype, const void* q, const float* w, const void* k, const float* k_scale, int T, int N, int H,
+                            int D, int topk, int causal_offset, const int32_t* sample_idx, int n_sample, int32_t* out_idx,
+                            float* out_score, void* workspace, size_t workspace_bytes, const lt_tunables* tunables,
+                            void* stream) {
+  if (sample_idx == nullptr || n_sample <= 0 || n_sample > LT_MAX_SAMPLE) return LT_ERR_INVALID_ARG;
+  return topk_impl(dtype, q, w, k, k_scale, T, N, H, D, topk, causal_offset, out_idx, out_score, workspace, workspace_bytes,
+                   tunables, static_cast<cudaStream_t>(stream), sample_idx, n_sample);
+}
+
+size_t lt_indexer_topk_sampled_workspace_bytes(int dtype, int T, int N, int H, int D, int topk, int n_sample,
+                                               const lt_tunables* tunables) {
+  if ((dtype != LT_DTYPE_F32 && dtype != LT_DTYPE_BF16 && dtype != LT_DTYPE_E4M3) || T <= 0 || N <= 0 || H <= 0 || D <= 0 ||
+      topk <= 0 || topk > N || topk > LT_MAX_TOPK || n_sample <= 0 || n_sample > LT_MAX_SAMPLE)
+    return 0;
+  const Tun tun = resolve_tunables(tunables);
+  return make_layout(use_fused(tun, dtype, H, D), T, N, topk, N - 1, tun, n_sample,
+                     static_cast<int>(static_cast<size_t>(D) * elem_bytes(dtype))).total;
+}
+
+size_t lt_topk_frequent_workspace_bytes(int N) {
+  if (N <= 0) return 0;
+  return align_up(static_cast<size_t>(N) * 4) + align_up(static_cast<size_t>(LT_MAX_TOPK) * 4);
+}
+
+int lt_topk_frequent(const int32_t* idx, int T, int topk, int N, int n_out, int32_t* out_pos, int32_t* out_count,
+                     void* workspace, size_t workspace_bytes, void* stream_) {
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  if (idx == nullptr || out_pos == nullptr || T <= 0 || topk <= 0 || N <= 0 || n_out <= 0 || n_out > N || n_out > LT_MAX_TOPK ||
+      T > (1 << 24))
+    return LT_ERR_INVALID_ARG;
+  if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) != 0 ||
+      workspace_bytes < lt_topk_frequent_workspace_bytes(N))
+    return LT_ERR_WORKSPACE;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  unsigned int* counts = reinterpret_cast<unsigned int*>(ws);
+  float* sel_score = reinterpret_cast<float*>(ws + align_up(static_cast<size_t>(N) * 4));
+  LT_CUDA(cudaMemsetAsync(counts, 0, static_cast<size_t>(N) * 4, stream));
+  LT_LAUNCH(launch_count_positions(idx, static_cast<long long>(T) * topk, N, counts, stream));
+  // a position occurs at most once per row, and in any case at most T * topk < 2^24 * 2^13 times; counts up
+  // to 2^24 are exact in fp32, larger ones (only possible with repeated positions inside a row) would still
+  // rank monotonically but lose their low bits, so such matrices are outside the contract
+  LT_LAUNCH(launch_counts_to_float(counts, N, stream));
+  SelectRowsParams sp{};
+  sp.scores = reinterpret_cast<const float*>(counts);
+  sp.ld = N;
+  sp.n_blocks = 1;
+  sp.row_begin = 0;
+  sp.T = 1;
+  sp.N = N;
+  sp.topk = n_out;
+  sp.causal_offset = N - 1;
+  sp.out_idx = out_pos;
+  sp.out_score = sel_score;
+  LT_LAUNCH(launch_select_rows(sp, stream));
+  if (out_count != nullptr) LT_LAUNCH(launch_float_to_counts(sel_score, n_out, out_count, stream));
+  return LT_OK;
 }
 
 int lt_indexer_sample_plan(int N, int topk, int causal_offset, const lt_tunables* tunables, int plan3[3]) {

@@ -99,4 +99,14 @@ struct SelectRowsParams {
 };
 cudaError_t launch_select_rows(const SelectRowsParams& p, cudaStream_t stream);
 
+// ---- lt_sampler.cu --------------------------------------------------------------------------
+// counts[p] += occurrences of p in idx[0..n) (entries outside [0, N) are skipped); counts must be zeroed.
+cudaError_t launch_count_positions(const int32_t* idx, long long n, int N, unsigned int* counts, cudaStream_t stream);
+// in place: counts[i] (u32) -> the same value as fp32 bits
+cudaError_t launch_counts_to_float(unsigned int* counts, int N, cudaStream_t stream);
+cudaError_t launch_float_to_counts(const float* f, int n, int32_t* out, cudaStream_t stream);
+// dense copy of the key rows (row_bytes each, multiple of 16) and scales at the sampled positions
+cudaError_t launch_gather_keys(const void* k, const float* k_scale, const int32_t* sample_idx, int n_sample, int N,
+                               int row_bytes, void* out_k, float* out_scale, cudaStream_t stream);
+
 }  // namespace lt

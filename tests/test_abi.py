@@ -56,6 +56,15 @@ def test_host_side_argument_checks(lib):
     # workspace too small / missing
     assert lib.lt_indexer_topk_ex(1, fake, fake, fake, null, 8, 64, 64, 128, 4, 56, fake, null, fake, 16, None, null) == -3
     assert lib.lt_indexer_topk_ex(1, fake, fake, fake, null, 8, 64, 64, 128, 4, 56, fake, null, null, 0, None, null) == -3
+    # sampled form: missing sample, sample too large
+    assert lib.lt_indexer_topk_sampled(1, fake, fake, fake, null, 8, 64, 64, 128, 4, 56, null, 8, fake, null, fake, 1 << 30, None, null) == -1
+    assert lib.lt_indexer_topk_sampled(1, fake, fake, fake, null, 8, 64, 64, 128, 4, 56, fake, 32769, fake, null, fake, 1 << 30, None, null) == -1
+    assert lib.lt_indexer_topk_sampled_workspace_bytes(1, 8, 64, 64, 128, 4, 0, None) == 0
+    assert lib.lt_indexer_topk_sampled_workspace_bytes(1, 8, 64, 64, 128, 4, 12, None) > lib.lt_indexer_topk_workspace_bytes(1, 8, 64, 64, 128, 4, None) - 4096
+    # frequency selector: sizes, workspace
+    assert lib.lt_topk_frequent(fake, 8, 4, 64, 65, fake, null, fake, 1 << 20, null) == -1
+    assert lib.lt_topk_frequent(fake, 8, 4, 64, 8, fake, null, fake, 16, null) == -3
+    assert lib.lt_topk_frequent_workspace_bytes(0) == 0 and lib.lt_topk_frequent_workspace_bytes(1000) >= 4000
     # the fused path cannot be forced onto a shape it does not support
     tun = binding.Tunables(path=binding.LT_PATH_FUSED)
     assert lib.lt_indexer_topk_ex(0, fake, fake, fake, null, 8, 64, 8, 64, 4, 56, fake, null, fake, 1 << 30,

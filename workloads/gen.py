@@ -8,6 +8,7 @@ structure follow the five benchmark configurations:
   dsa_bf16      bf16 q/k, keys carry a slow positional drift along one direction
   fp8_ar1       e4m3 codes + per-token fp32 absmax scales, AR(1) queries (rho = 0.9)
   fp8_1m        same recipe, 4096 queries at the end of a 1,048,576-key context
+  hot_fp8       e4m3, a shared set of high-scoring keys (for the previous-chunk sampler)
   adv_planted   heavy-tailed key norms + 5 % planted keys along query directions
   adv_cluster   all planted keys identical, along a component shared by all queries
   adv_ties      q/k coordinates on 4 levels (continuous head weights)
@@ -151,6 +152,8 @@ CONFIGS = {
     "adv_cluster": ("cluster", "bf16", 4096, 65536, 64, 128, 2048, 6),
     "adv_ties": ("ties", "bf16", 4096, 65536, 64, 128, 2048, 7),
     "adv_ties_exact": ("ties_exact", "bf16", 4096, 65536, 64, 128, 2048, 8),
+    # stand-in for the cross-chunk structure the previous-chunk sampler relies on (paper Sec. 3.2 "Sampling")
+    "hot_fp8": ("hot", "e4m3", 4096, 1048576, 64, 128, 2048, 9),
 }
 
 
@@ -180,6 +183,20 @@ def make_inputs(recipe: str, dtype: str, T: int, N: int, H: int, D: int, topk: i
 
     if recipe in ("iid", "ar1"):
         k = _normal(seed, 1, (N, D), sd)
+    elif recipe == "hot":
+        # "adjacent chunks attend to the same prefix tokens": 3k/2 keys at random positions of the first half of the
+        # context carry a shared direction c that every query head carries too, and the head weights are
+        # positive, so these keys score high for every row of every chunk; which of them make a row's top-k
+        # is decided by the independent parts
+        k = _normal(seed, 1, (N, D), sd)
+        c = _unit(_normal(seed, 6, (D,), 1.0))
+        n_hot = min(max(N // 8, 1), (3 * topk) // 2)
+        pos = np.sort(_rng(seed, 5).permutation(max(N // 2, n_hot))[:n_hot])
+        k[pos] += c[None, :]
+        q = q + np.float32(0.5) * c[None, None, :]
+        w = np.abs(w)
+        meta["hot_pos"] = pos
+        meta["hot_dir"] = c
     elif recipe == "drift":
         k = _normal(seed, 1, (N, D), sd)
         u = _unit(_normal(seed, 3, (D,), 1.0))
