@@ -15,6 +15,7 @@ namespace lt {
 namespace {
 
 constexpr int kSelThreads = 1024;
+constexpr int kSelBatch = 8;  // independent row loads in flight per thread of the full-row select
 constexpr int kSelCap = 2 * LT_MAX_TOPK;  // 64-bit keys the final select can sort in shared memory
 
 // ---------------------------------------------------------------------------------------------
@@ -252,7 +253,7 @@ __global__ void __launch_bounds__(kFinalThreads) final_select_kernel(const Final
 __global__ void __launch_bounds__(kSelThreads) select_rows_kernel(const SelectRowsParams p) {
   extern __shared__ uint64_t sel[];  // LT_MAX_TOPK keys
   __shared__ unsigned int hist[256];
-  __shared__ unsigned int s_prefix, s_remaining, s_gt, s_eq_base;
+  __shared__ unsigned int s_prefix, s_remaining, s_gt;
   __shared__ unsigned int warp_cnt[32];
   int t;
   if (p.fb_list != nullptr) {
@@ -288,10 +289,37 @@ __global__ void __launch_bounds__(kSelThreads) select_rows_kernel(const SelectRo
     if (tid < 256) hist[tid] = 0;
     __syncthreads();
     const unsigned int prefix = s_prefix;
-    for (int i = tid; i < vis; i += kSelThreads) {
-      unsigned int key = score_to_key(__float_as_uint(row[i]));
-      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+    // Scores of one row share their leading bits, so consecutive candidates of a thread mostly want the
+    // same counter: each thread run-length-encodes its digits and issues one atomic per run.
+    unsigned int run_digit = 0x100u, run_len = 0;
+    // (kSelBatch loads in flight per thread: one row is read by one SM, which is latency-bound otherwise)
+    for (int base = 0; base < vis; base += kSelThreads * kSelBatch) {
+      float v[kSelBatch];
+#pragma unroll
+      for (int j = 0; j < kSelBatch; ++j) {
+        const int i = base + j * kSelThreads + tid;
+        v[j] = i < vis ? row[i] : 0.f;
+      }
+#pragma unroll
+      for (int j = 0; j < kSelBatch; ++j) {
+        const int i = base + j * kSelThreads + tid;
+        unsigned int digit = 0x100u;  // "not a candidate" (out of range or another prefix)
+        if (i < vis) {
+          const unsigned int key = score_to_key(__float_as_uint(v[j]));
+          if ((key & mask) == prefix) digit = (key >> shift) & 255u;
+        }
+        if (digit < 0x100u) {
+          if (digit == run_digit) {
+            ++run_len;
+          } else {
+            if (run_len > 0) atomicAdd(&hist[run_digit], run_len);
+            run_digit = digit;
+            run_len = 1;
+          }
+        }
+      }
     }
+    if (run_len > 0) atomicAdd(&hist[run_digit], run_len);
     __syncthreads();
     if (tid == 0) {
       unsigned int remaining = s_remaining, cum = 0;
@@ -313,43 +341,66 @@ __global__ void __launch_bounds__(kSelThreads) select_rows_kernel(const SelectRo
   const unsigned int kth = s_prefix;                 // key of the k-th largest score
   const unsigned int need_eq = s_remaining;          // how many keys equal to it are selected
   const unsigned int n_gt = static_cast<unsigned int>(kk) - need_eq;
-  if (tid == 0) {
-    s_gt = 0;
-    s_eq_base = 0;
+  if (tid == 0) s_gt = 0;
+  // Collection.  Keys above the k-th go in any order (the sort follows).  Ties at the k-th value keep
+  // the lowest indices, so they are ranked in index order: every warp owns one contiguous range of the
+  // row, counts its ties, and after one prefix sum over the 32 warps writes them at their ranks.
+  const int per_warp = (((vis + 31) / 32 + 31) / 32) * 32;  // range length: a multiple of 32 covering vis / 32
+  const int lo = wid * per_warp;
+  const int hi = min(vis, lo + per_warp);
+  unsigned int my_eq = 0;
+  for (int base = lo; base < hi; base += 32 * kSelBatch) {
+    float v[kSelBatch];
+#pragma unroll
+    for (int j = 0; j < kSelBatch; ++j) {
+      const int i = base + j * 32 + lane;
+      v[j] = i < hi ? row[i] : 0.f;
+    }
+#pragma unroll
+    for (int j = 0; j < kSelBatch; ++j) {
+      const int i = base + j * 32 + lane;
+      const bool eq = i < hi && score_to_key(__float_as_uint(v[j])) == kth;
+      my_eq += __popc(__ballot_sync(0xffffffffu, eq));
+    }
   }
+  if (lane == 0) warp_cnt[wid] = my_eq;
   __syncthreads();
-  for (int base = 0; base < vis; base += kSelThreads) {
-    const int i = base + tid;
+  unsigned int running = 0;
+  for (int wq = 0; wq < wid; ++wq) running += warp_cnt[wq];
+  for (int base0 = lo; base0 < hi; base0 += 32 * kSelBatch) {
+   float v[kSelBatch];
+#pragma unroll
+   for (int j = 0; j < kSelBatch; ++j) {
+     const int i = base0 + j * 32 + lane;
+     v[j] = i < hi ? row[i] : 0.f;
+   }
+#pragma unroll
+   for (int j = 0; j < kSelBatch; ++j) {
+    const int i = base0 + j * 32 + lane;
     unsigned int key = 0;
     bool gt = false, eq = false;
-    if (i < vis) {
-      key = score_to_key(__float_as_uint(row[i]));
+    if (i < hi) {
+      key = score_to_key(__float_as_uint(v[j]));
       gt = key > kth;
       eq = key == kth;
     }
-    if (gt) {
-      unsigned int pos = atomicAdd(&s_gt, 1u);
-      sel[pos] = (static_cast<uint64_t>(key) << 32) | (0xffffffffu - static_cast<unsigned int>(i));
+    const uint64_t packed = (static_cast<uint64_t>(key) << 32) | (0xffffffffu - static_cast<unsigned int>(i));
+    const unsigned int gt_ballot = __ballot_sync(0xffffffffu, gt);
+    if (gt_ballot != 0) {
+      unsigned int pos = 0;
+      if (lane == 0) pos = atomicAdd(&s_gt, static_cast<unsigned int>(__popc(gt_ballot)));
+      pos = __shfl_sync(0xffffffffu, pos, 0);
+      if (gt) sel[pos + __popc(gt_ballot & ((1u << lane) - 1u))] = packed;
     }
-    // ties at the k-th value: keep the lowest indices, so rank them in index order
     const unsigned int eq_ballot = __ballot_sync(0xffffffffu, eq);
-    if (lane == 0) warp_cnt[wid] = __popc(eq_ballot);
-    __syncthreads();
-    const unsigned int eq_base = s_eq_base;
-    unsigned int before = 0, total = 0;
-    for (int wq = 0; wq < 32; ++wq) {
-      unsigned int c = warp_cnt[wq];
-      if (wq < wid) before += c;
-      total += c;
-    }
     if (eq) {
-      unsigned int rank = eq_base + before + __popc(eq_ballot & ((1u << lane) - 1u));
-      if (rank < need_eq) sel[n_gt + rank] = (static_cast<uint64_t>(key) << 32) | (0xffffffffu - static_cast<unsigned int>(i));
+      const unsigned int rank = running + __popc(eq_ballot & ((1u << lane) - 1u));
+      if (rank < need_eq) sel[n_gt + rank] = packed;
     }
-    __syncthreads();
-    if (tid == 0) s_eq_base = eq_base + total;
-    __syncthreads();
+    running += __popc(eq_ballot);
+   }
   }
+  __syncthreads();
   sort_and_write(sel, kk, p.topk, out_idx, out_score);
 }
 
