@@ -371,3 +371,56 @@ def test_frequent_positions_closed_form_and_invariants():
     assert frequent_positions(shuffled, 200, 48)[0].tolist() == pos.tolist()
     with pytest.raises(ValueError):
         frequent_positions(idx, 100, 10)
+
+
+# ---------------------------------------------------------------------------------------------
+# LiteDSA union list + membership masks (paper Sec. 3.3)
+# ---------------------------------------------------------------------------------------------
+
+def test_union_and_masks_match_set_brute_force():
+    from oracle import pack_mask_words, union_and_masks
+
+    rng = np.random.default_rng(21)
+    for trial in range(30):
+        N = int(rng.integers(4, 80))
+        T = int(rng.integers(1, 14))
+        k = int(rng.integers(1, min(N, 10) + 1))
+        group = int(rng.integers(1, 6))
+        idx = np.stack([rng.permutation(N)[:k] for _ in range(T)]).astype(np.int64)
+        idx[rng.random(idx.shape) < 0.15] = -1
+        unions, masks = union_and_masks(idx, N, group)
+        assert len(unions) == -(-T // group) and len(masks) == T
+        for g, u in enumerate(unions):
+            rows = range(g * group, min(T, (g + 1) * group))
+            want = sorted(set(int(v) for t in rows for v in idx[t] if v >= 0))
+            assert u.tolist() == want
+            acc = np.zeros(len(want), dtype=bool)
+            for t in rows:
+                mine = set(int(v) for v in idx[t] if v >= 0)
+                assert [want[s] for s in np.flatnonzero(masks[t])] == sorted(mine)
+                acc |= masks[t]
+                words = pack_mask_words(masks[t], (group * k + 31) // 32)
+                for s in range(len(want)):
+                    assert bool((int(words[s // 32]) >> (s % 32)) & 1) == bool(masks[t][s])
+                assert all(int(w) == 0 for w in words[(len(want) + 31) // 32:])
+            assert acc.all()  # every union entry belongs to at least one row
+
+
+def test_union_and_masks_closed_form():
+    from oracle import union_and_masks
+
+    # row t selects the multiples of (t + 1) below 60; a group of all rows -> union = every position that is a
+    # multiple of something in 1..T = everything from 0 to 59; one group per row -> the row's own list, full mask
+    T, N = 5, 60
+    width = N
+    idx = np.full((T, width), -1, dtype=np.int64)
+    for t in range(T):
+        m = np.arange(0, N, t + 1)
+        idx[t, :m.size] = m
+    unions, masks = union_and_masks(idx, N, T)
+    assert unions[0].tolist() == list(range(N))
+    for t in range(T):
+        assert np.flatnonzero(masks[t]).tolist() == list(range(0, N, t + 1))
+    unions, masks = union_and_masks(idx, N, 1)
+    for t in range(T):
+        assert unions[t].tolist() == list(range(0, N, t + 1)) and masks[t].all()
