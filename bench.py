@@ -195,6 +195,46 @@ def run_reference(args, rank: int):
     print(json.dumps(line))
 
 
+def time_aux_ops(torch, lt, out_idx, inp, hbm_gbs, peak_kind, reps=5):
+    """HBM-bound integer ops that consume a chunk's top-k matrix; algorithmic bytes = the index matrix once + outputs."""
+    def timed(fn):
+        fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(torch.cuda.current_stream())
+        for _ in range(reps):
+            fn()
+        e1.record(torch.cuda.current_stream())
+        e1.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    T, k, N = inp.T, inp.topk, inp.N
+    out = {}
+    n_out = min(3 * k, lt.LT_MAX_TOPK, N)
+    pos = torch.empty(n_out, dtype=torch.int32, device="cuda")
+    ws = torch.empty(lt.lt_topk_frequent_workspace_bytes(N), dtype=torch.uint8, device="cuda")
+    ms = timed(lambda: lt.lt_topk_frequent(out_idx, N, pos, None, ws))
+    nbytes = T * k * 4 + N * 4 + n_out * 4  # index matrix once, counts written once, result
+    out["lt_topk_frequent"] = {"ms": ms, "algorithmic_bytes": nbytes, "gbs": nbytes / ms / 1e6,
+                               "frac_of_hbm_peak": nbytes / ms / 1e6 / hbm_gbs, "peak_kind": peak_kind, "n_out": n_out}
+    group = 64
+    n_groups = -(-T // group)
+    cap = group * k
+    upos = torch.empty((n_groups, cap), dtype=torch.int32, device="cuda")
+    ulen = torch.empty(n_groups, dtype=torch.int32, device="cuda")
+    mask = torch.empty((T, (cap + 31) // 32), dtype=torch.int32, device="cuda")
+    ms = timed(lambda: lt.lt_dsa_union_mask(out_idx, N, group, upos, ulen, mask))
+    n_union = int(ulen.sum().item())
+    # index matrix once + the union entries + one mask bit per (row, union slot of its group), without the
+    # clearing of the full-capacity outputs (which the call does with two memsets and which is what dominates)
+    nbytes = T * k * 4 + n_union * 4 + sum(int(n) for n in ulen.tolist()) * group // 8
+    cleared = upos.numel() * 4 + mask.numel() * 4
+    out["lt_dsa_union_mask"] = {"ms": ms, "group": group, "mean_union_len": n_union / n_groups, "algorithmic_bytes": nbytes,
+                                "cleared_bytes": cleared, "gbs": nbytes / ms / 1e6, "gbs_with_clears": (nbytes + cleared) / ms / 1e6,
+                                "frac_of_hbm_peak": nbytes / ms / 1e6 / hbm_gbs, "peak_kind": peak_kind}
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -207,6 +247,9 @@ def main():
     ap.add_argument("--sampler", default="strided", choices=["strided", "prev_chunk"],
                     help="prev_chunk: the sample is the 3k most frequent top-k positions of the previous chunk "
                          "(computed untimed through lt_topk_frequent; paper Sec. 3.2 'Sampling')")
+    ap.add_argument("--aux", action="store_true",
+                    help="also time the auxiliary integer ops on this step's top-k result: lt_topk_frequent and "
+                         "lt_dsa_union_mask (group 64); adds an 'aux' object to the JSON line")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-unfused", action="store_true")
     ap.add_argument("--unfused-budget-mb", type=int, default=2048, help="score-matrix budget of the unfused GPU baseline")
@@ -393,6 +436,9 @@ def main():
         "status": {"bits": status[0], "fallback_rows": status[1], "max_survivors_per_row": status[2],
                    "mean_survivors_per_row": status[3] / inp.T, "overflow_rows": status[4]},
     }
+
+    if args.aux:
+        line["aux"] = time_aux_ops(torch, lt, out_idx, inp, peaks["hbm_gbs"], peak_kind)
 
     if not args.no_unfused:
         # in-repo unfused GPU baseline: dense scores to HBM in row sub-chunks, then a full-row radix select

@@ -165,6 +165,21 @@ int lt_topk_frequent(const int32_t* idx, int T, int topk, int N, int n_out, int3
 size_t lt_topk_frequent_workspace_bytes(int N);
 
 /*
+ * LiteDSA union list and membership masks (paper Sec. 3.3 "LiteDSA").  Rows are taken in consecutive
+ * groups of `group` (the last group may be shorter).  For group g:
+ *   union_pos[g][0 .. union_len[g])  the distinct positions selected by any row of the group, ascending
+ *                                    (what a sweep of the group's bitmap yields); the rest of the
+ *                                    group * topk slots is -1
+ *   member_mask[t][s / 32] bit s % 32 = 1 iff union_pos[g(t)][s] is one of idx[t][:]
+ * All pointers are device memory: idx [T][topk] int32 (entries < 0 or >= N are skipped), union_pos
+ * [ceil(T / group)][group * topk] int32, union_len [ceil(T / group)] int32, member_mask
+ * [T][ceil(group * topk / 32)] uint32.  1 <= group, group * topk <= 2^24.  Integer work only: the
+ * result is exact.  The masked attention that consumes these is not part of this library.
+ */
+int lt_dsa_union_mask(const int32_t* idx, int T, int topk, int N, int group,
+                      int32_t* union_pos, int32_t* union_len, uint32_t* member_mask, void* stream);
+
+/*
  * Host-only helper (no GPU work): the sample plan the fused path would use for this problem.
  * plan3[0] = sample size k', plan3[1] = stride between sampled key positions (the sample is
  * positions 0, stride, 2 stride, ... of the keys every row of the chunk can see), plan3[2] = rank r

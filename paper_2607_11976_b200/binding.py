@@ -70,6 +70,8 @@ def load() -> ctypes.CDLL:
     lib.lt_topk_frequent.restype = i
     lib.lt_topk_frequent_workspace_bytes.argtypes = [i]
     lib.lt_topk_frequent_workspace_bytes.restype = sz
+    lib.lt_dsa_union_mask.argtypes = [ip, i, i, i, i, ip, ip, vp, vp]
+    lib.lt_dsa_union_mask.restype = i
     lib.lt_indexer_sample_plan.argtypes = [i, i, i, ctypes.POINTER(Tunables), ctypes.POINTER(ctypes.c_int)]
     lib.lt_indexer_sample_plan.restype = i
     lib.lt_indexer_scores.argtypes = [i, vp, fp, vp, fp, i, i, i, i, i, i, i, fp, i, vp]
@@ -185,6 +187,13 @@ def lt_topk_frequent(idx, N: int, out_pos, out_count, workspace, stream=None) ->
     T, topk = idx.shape
     _check(load().lt_topk_frequent(_ptr(idx), T, topk, N, out_pos.numel(), _ptr(out_pos), _ptr(out_count), _ptr(workspace),
                                    workspace.numel() * workspace.element_size(), _stream(stream)), "lt_topk_frequent")
+
+
+def lt_dsa_union_mask(idx, N: int, group: int, union_pos, union_len, member_mask, stream=None) -> None:
+    """LiteDSA union list + membership masks of consecutive groups of `group` rows of the [T, topk] matrix idx."""
+    T, topk = idx.shape
+    _check(load().lt_dsa_union_mask(_ptr(idx), T, topk, N, group, _ptr(union_pos), _ptr(union_len), _ptr(member_mask),
+                                    _stream(stream)), "lt_dsa_union_mask")
 
 
 def lt_indexer_scores(dtype, q, w, k, k_scale, causal_offset: int, row_begin: int, row_end: int, out_scores,

@@ -525,6 +525,15 @@ int lt_topk_frequent(const int32_t* idx, int T, int topk, int N, int n_out, int3
   return LT_OK;
 }
 
+int lt_dsa_union_mask(const int32_t* idx, int T, int topk, int N, int group, int32_t* union_pos, int32_t* union_len,
+                      uint32_t* member_mask, void* stream) {
+  if (idx == nullptr || union_pos == nullptr || union_len == nullptr || member_mask == nullptr || T <= 0 || topk <= 0 || N <= 0 ||
+      group <= 0 || static_cast<long long>(group) * topk > (1ll << 24))
+    return LT_ERR_INVALID_ARG;
+  LT_LAUNCH(launch_dsa_union(idx, T, topk, N, group, union_pos, union_len, member_mask, static_cast<cudaStream_t>(stream)));
+  return LT_OK;
+}
+
 int lt_indexer_sample_plan(int N, int topk, int causal_offset, const lt_tunables* tunables, int plan3[3]) {
   if (plan3 == nullptr || N <= 0 || topk <= 0 || topk > N || topk > LT_MAX_TOPK) return LT_ERR_INVALID_ARG;
   const Layout L = make_layout(true, 1, N, topk, causal_offset, resolve_tunables(tunables));

@@ -109,4 +109,10 @@ cudaError_t launch_float_to_counts(const float* f, int n, int32_t* out, cudaStre
 cudaError_t launch_gather_keys(const void* k, const float* k_scale, const int32_t* sample_idx, int n_sample, int N,
                                int row_bytes, void* out_k, float* out_scale, cudaStream_t stream);
 
+// ---- lt_dsa_union.cu ------------------------------------------------------------------------
+// LiteDSA union list + membership masks of consecutive groups of `group` rows (paper Sec. 3.3).
+// union_pos [n_groups][group * topk] (-1 beyond union_len), mask [T][ceil(group * topk / 32)].
+cudaError_t launch_dsa_union(const int32_t* idx, int T, int topk, int N, int group, int32_t* union_pos, int32_t* union_len,
+                             uint32_t* mask, cudaStream_t stream);
+
 }  // namespace lt

@@ -65,6 +65,9 @@ def test_host_side_argument_checks(lib):
     assert lib.lt_topk_frequent(fake, 8, 4, 64, 65, fake, null, fake, 1 << 20, null) == -1
     assert lib.lt_topk_frequent(fake, 8, 4, 64, 8, fake, null, fake, 16, null) == -3
     assert lib.lt_topk_frequent_workspace_bytes(0) == 0 and lib.lt_topk_frequent_workspace_bytes(1000) >= 4000
+    # LiteDSA union builder: group size, slot limit
+    assert lib.lt_dsa_union_mask(fake, 8, 4, 64, 0, fake, fake, fake, null) == -1
+    assert lib.lt_dsa_union_mask(fake, 8, 8192, 1 << 20, 4096, fake, fake, fake, null) == -1
     # the fused path cannot be forced onto a shape it does not support
     tun = binding.Tunables(path=binding.LT_PATH_FUSED)
     assert lib.lt_indexer_topk_ex(0, fake, fake, fake, null, 8, 64, 8, 64, 4, 56, fake, null, fake, 1 << 30,
