@@ -69,20 +69,22 @@ __device__ __forceinline__ int bin_of(float s, float smin, float width) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// bitonic sort of n (power of two) 64-bit keys in shared memory, descending.
+// bitonic sort of n (power of two, >= 2) 64-bit keys in shared memory, descending.  Every thread
+// handles whole compare-exchange pairs: pair t of a stage with distance j is (i, i | j) where i is t
+// with a zero bit inserted at bit log2(j), so no thread idles on the upper element of a pair.
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ void bitonic_sort_desc(uint64_t* s, int n, int tid, int nthreads) {
+  const int half = n >> 1;
   for (int k = 2; k <= n; k <<= 1) {
     for (int j = k >> 1; j > 0; j >>= 1) {
-      for (int i = tid; i < n; i += nthreads) {
-        int ixj = i ^ j;
-        if (ixj > i) {
-          uint64_t a = s[i], b = s[ixj];
-          bool desc = (i & k) == 0;
-          if (desc ? (a < b) : (a > b)) {
-            s[i] = b;
-            s[ixj] = a;
-          }
+      for (int t = tid; t < half; t += nthreads) {
+        const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+        const int ixj = i | j;
+        const uint64_t a = s[i], b = s[ixj];
+        const bool desc = (i & k) == 0;
+        if (desc ? (a < b) : (a > b)) {
+          s[i] = b;
+          s[ixj] = a;
         }
       }
       __syncthreads();
