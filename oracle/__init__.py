@@ -13,3 +13,4 @@ from .indexer_topk import (  # noqa: F401
 )
 from .sampler import frequent_positions, position_counts  # noqa: F401,E402
 from .litedsa import pack_mask_words, union_and_masks  # noqa: F401,E402
+from .knn import knn_scores, knn_topk  # noqa: F401,E402

@@ -424,3 +424,49 @@ def test_union_and_masks_closed_form():
     unions, masks = union_and_masks(idx, N, 1)
     for t in range(T):
         assert unions[t].tolist() == list(range(0, N, t + 1)) and masks[t].all()
+
+
+# ---------------------------------------------------------------------------------------------
+# k-NN (inner-product) variant: Eq. 2 with f(q, x) = q . x over the whole corpus
+# ---------------------------------------------------------------------------------------------
+
+def test_knn_oracle_matches_exact_rational_brute_force():
+    from fractions import Fraction
+
+    from oracle import decode_bf16, knn_topk
+    from workloads import bf16_encode
+
+    rng = np.random.default_rng(31)
+    for trial in range(6):
+        T, N, D, k = int(rng.integers(1, 4)), int(rng.integers(3, 20)), int(rng.integers(1, 9)), 3
+        q = bf16_encode(rng.standard_normal((T, D)).astype(np.float32))
+        x = bf16_encode(rng.standard_normal((N, D)).astype(np.float32))
+        if trial == 0:
+            x[1] = x[0]  # an exact tie: the lower index must win
+        qf = [[Fraction(float(v)) for v in row] for row in decode_bf16(q)]
+        xf = [[Fraction(float(v)) for v in row] for row in decode_bf16(x)]
+        idx, val, rms, full = knn_topk(q, x, min(k, N))
+        for t in range(T):
+            scores = [sum(a * b for a, b in zip(qf[t], xv)) for xv in xf]
+            order = sorted(range(N), key=lambda s: (-scores[s], s))[:min(k, N)]
+            assert idx[t].tolist() == order
+            assert all(abs(Fraction(float(val[t][j])) - scores[order[j]]) <= Fraction(1, 10 ** 12) for j in range(len(order)))
+
+
+def test_knn_oracle_agrees_with_indexer_oracle_where_relu_is_identity():
+    # H = 1, w = 1, non-negative coordinates: every dot product is >= 0, so Eq. 1 reduces to the inner product
+    from oracle import indexer_topk, knn_topk
+    from workloads import bf16_encode
+
+    rng = np.random.default_rng(32)
+    T, N, D, k = 5, 300, 16, 40
+    q = bf16_encode(np.abs(rng.standard_normal((T, D))).astype(np.float32))
+    x = bf16_encode(np.abs(rng.standard_normal((N, D))).astype(np.float32))
+    idx, val, _, _ = knn_topk(q, x, k)
+    ref = indexer_topk(q.reshape(T, 1, D), np.ones((T, 1), dtype=np.float32), x, None, "bf16", k, N)  # every key visible
+    assert np.array_equal(idx, ref.idx) and np.allclose(val, ref.score, rtol=0, atol=1e-12)
+    # scaling a query by a power of two scales its scores exactly and keeps the selected set
+    from oracle import decode_bf16
+    q2 = bf16_encode(decode_bf16(q).astype(np.float32) * np.float32(4.0))
+    idx2, val2, _, _ = knn_topk(q2, x, k)
+    assert np.array_equal(idx2, idx) and np.array_equal(val2, 4.0 * val)

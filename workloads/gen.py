@@ -260,3 +260,65 @@ def make_config(name: str, T: Optional[int] = None, N: Optional[int] = None, H: 
     recipe, dt, T0, N0, H0, D0, k0, cid = CONFIGS[name]
     return make_inputs(recipe, dtype or dt, T or T0, N or N0, H or H0, D or D0, topk or k0,
                        seed if seed is not None else BASE_SEED + cid, causal_offset, name=name)
+
+
+# ----------------------------------------------------------------------------
+# k-NN retrieval variant (inner product over a corpus of embeddings)
+# ----------------------------------------------------------------------------
+
+@dataclasses.dataclass
+class KnnInputs:
+    """A batch of queries and a corpus, both bf16 codes (uint16), row-major [rows, D]."""
+
+    name: str
+    q: np.ndarray      # [T, D] uint16
+    x: np.ndarray      # [N, D] uint16
+    topk: int
+    meta: dict
+
+    @property
+    def T(self) -> int:
+        return int(self.q.shape[0])
+
+    @property
+    def N(self) -> int:
+        return int(self.x.shape[0])
+
+    @property
+    def D(self) -> int:
+        return int(self.q.shape[1])
+
+    def valid_pairs(self) -> int:
+        return self.T * self.N
+
+
+KNN_CONFIGS = {
+    # name: (T, N, D, topk, config id for the seed).  Stand-in for 768-d passage embeddings: unit vectors drawn
+    # around 64 cluster centres (concentrated similarities, no temporal structure), queries drawn like passages.
+    "knn_bf16": (64, 1 << 20, 768, 1024, 20),
+}
+
+
+def make_knn(name: str = "knn_bf16", T: Optional[int] = None, N: Optional[int] = None, D: Optional[int] = None,
+             topk: Optional[int] = None) -> KnnInputs:
+    T0, N0, D0, k0, cid = KNN_CONFIGS[name]
+    T, N, D, topk = T or T0, N or N0, D or D0, topk or k0
+    seed = BASE_SEED + cid
+    n_centres = 64
+    centres = _unit(_normal(seed, 0, (n_centres, D), 1.0))
+
+    def draw(stream: int, rows: int) -> np.ndarray:
+        which = _rng(seed, stream).integers(0, n_centres, size=rows)
+        out = np.empty((rows, D), dtype=np.float32)
+        step = 1 << 16
+        for r0 in range(0, rows, step):  # in slabs: the corpus can be several GB in fp32
+            r1 = min(rows, r0 + step)
+            g = _rng(seed, stream + 100 + r0 // step).standard_normal((r1 - r0, D), dtype=np.float32)
+            out[r0:r1] = _unit(g / np.float32(np.sqrt(D)) + np.float32(0.7) * centres[which[r0:r1]])
+        return out
+
+    x = draw(1, N)
+    q = draw(2, T)
+    return KnnInputs(name=name, q=bf16_encode(q), x=bf16_encode(x), topk=topk,
+                     meta={"recipe": "embed", "seed": seed, "centres": n_centres})
+
