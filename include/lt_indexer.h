@@ -165,6 +165,31 @@ int lt_topk_frequent(const int32_t* idx, int T, int topk, int N, int n_out, int3
 size_t lt_topk_frequent_workspace_bytes(int N);
 
 /*
+ * k-NN (inner-product) variant: exact top-k of f(q, x) = q . x over a whole corpus for a batch of
+ * queries (paper Sec. 3.1, Eq. 2; the retrieval workload of Sec. 4.1: 768-d embeddings, batches of 64
+ * queries, k up to 8192, no causal mask).  Same method as the indexer path - strided sample, bins,
+ * online threshold, filtered write-back, exact final select, exact fallback - with the scores coming
+ * straight from the tensor cores (Sec. 3.2 "Filtering", first case), so the corpus is streamed from
+ * HBM once per 64 queries.
+ *   dtype       LT_DTYPE_BF16 only
+ *   q           device, [T][D] bf16;  x: device, [N][D] bf16 (both 16-byte aligned, row-major, dense)
+ *   D           a multiple of 64, at most 768;  topk: 1 .. min(N, LT_MAX_TOPK)
+ *   out_idx     device, [T][topk] int32 in (score descending, index ascending) order; out_score: device,
+ *               [T][topk] fp32 or NULL
+ *   workspace   device, 256-byte aligned, at least lt_knn_topk_workspace_bytes(...) bytes; holds the
+ *               status block (lt_read_status)
+ * lt_knn_scores writes the dense scores of rows [row_begin, row_end) to out_scores[(t - row_begin) * N + s],
+ * bit-identical to the scores lt_knn_topk ranks (debugging and parity).
+ * Errors: LT_ERR_UNSUPPORTED for another dtype or D, LT_ERR_INVALID_ARG, LT_ERR_WORKSPACE, LT_ERR_CUDA.
+ */
+int lt_knn_topk(int dtype, const void* q, const void* x, int T, int N, int D, int topk,
+                int32_t* out_idx, float* out_score,
+                void* workspace, size_t workspace_bytes, const lt_tunables* tunables, void* stream);
+size_t lt_knn_topk_workspace_bytes(int dtype, int T, int N, int D, int topk, const lt_tunables* tunables);
+int lt_knn_scores(int dtype, const void* q, const void* x, int T, int N, int D,
+                  int row_begin, int row_end, float* out_scores, void* stream);
+
+/*
  * LiteDSA union list and membership masks (paper Sec. 3.3 "LiteDSA").  Rows are taken in consecutive
  * groups of `group` (the last group may be shorter).  For group g:
  *   union_pos[g][0 .. union_len[g])  the distinct positions selected by any row of the group, ascending

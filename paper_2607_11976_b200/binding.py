@@ -70,6 +70,12 @@ def load() -> ctypes.CDLL:
     lib.lt_topk_frequent.restype = i
     lib.lt_topk_frequent_workspace_bytes.argtypes = [i]
     lib.lt_topk_frequent_workspace_bytes.restype = sz
+    lib.lt_knn_topk.argtypes = [i, vp, vp, i, i, i, i, ip, fp, vp, sz, ctypes.POINTER(Tunables), vp]
+    lib.lt_knn_topk.restype = i
+    lib.lt_knn_topk_workspace_bytes.argtypes = [i, i, i, i, i, ctypes.POINTER(Tunables)]
+    lib.lt_knn_topk_workspace_bytes.restype = sz
+    lib.lt_knn_scores.argtypes = [i, vp, vp, i, i, i, i, i, fp, vp]
+    lib.lt_knn_scores.restype = i
     lib.lt_dsa_union_mask.argtypes = [ip, i, i, i, i, ip, ip, vp, vp]
     lib.lt_dsa_union_mask.restype = i
     lib.lt_indexer_sample_plan.argtypes = [i, i, i, ctypes.POINTER(Tunables), ctypes.POINTER(ctypes.c_int)]
@@ -187,6 +193,28 @@ def lt_topk_frequent(idx, N: int, out_pos, out_count, workspace, stream=None) ->
     T, topk = idx.shape
     _check(load().lt_topk_frequent(_ptr(idx), T, topk, N, out_pos.numel(), _ptr(out_pos), _ptr(out_count), _ptr(workspace),
                                    workspace.numel() * workspace.element_size(), _stream(stream)), "lt_topk_frequent")
+
+
+def lt_knn_topk_workspace_bytes(T: int, N: int, D: int, topk: int, tunables: Optional[Tunables] = None) -> int:
+    return int(load().lt_knn_topk_workspace_bytes(LT_DTYPE_BF16, T, N, D, topk, ctypes.byref(tunables) if tunables else None))
+
+
+def lt_knn_topk(q, x, topk: int, out_idx, out_score, workspace, tunables: Optional[Tunables] = None, stream=None) -> None:
+    """Exact top-k inner products of the bf16 queries q [T, D] over the bf16 corpus x [N, D]."""
+    T, D = q.shape
+    N, D2 = x.shape
+    if D2 != D:
+        raise ValueError("q and x disagree on D")
+    _check(load().lt_knn_topk(LT_DTYPE_BF16, _ptr(q), _ptr(x), T, N, D, topk, _ptr(out_idx), _ptr(out_score), _ptr(workspace),
+                              workspace.numel() * workspace.element_size(), ctypes.byref(tunables) if tunables else None,
+                              _stream(stream)), "lt_knn_topk")
+
+
+def lt_knn_scores(q, x, row_begin: int, row_end: int, out_scores, stream=None) -> None:
+    T, D = q.shape
+    N = x.shape[0]
+    _check(load().lt_knn_scores(LT_DTYPE_BF16, _ptr(q), _ptr(x), T, N, D, row_begin, row_end, _ptr(out_scores), _stream(stream)),
+           "lt_knn_scores")
 
 
 def lt_dsa_union_mask(idx, N: int, group: int, union_pos, union_len, member_mask, stream=None) -> None:

@@ -616,6 +616,183 @@ int lt_indexer_scores(int dtype, const void* q, const float* w, const void* k, c
   return LT_OK;
 }
 
+// ---- k-NN (inner-product) variant --------------------------------------------------------------
+namespace {
+
+int knn_check(int dtype, const void* q, const void* x, int T, int N, int D) {
+  if (dtype != LT_DTYPE_BF16) return LT_ERR_UNSUPPORTED;
+  if (q == nullptr || x == nullptr || T <= 0 || N <= 0 || D <= 0) return LT_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(x)) return LT_ERR_INVALID_ARG;
+  if (!scan_knn_supported(D)) return LT_ERR_UNSUPPORTED;
+  return LT_OK;
+}
+
+int knn_seg_tiles(const Tun& tun, int n_keys, int grid) {
+  if (tun.segment_tiles > 0) return tun.segment_tiles;
+  const int n_tiles = (n_keys + kTileKeys - 1) / kTileKeys;
+  int seg = 32;
+  while (seg > 2 && (n_tiles + seg - 1) / seg < 4 * grid) seg >>= 1;
+  return seg;
+}
+
+}  // namespace
+
+size_t lt_knn_topk_workspace_bytes(int dtype, int T, int N, int D, int topk, const lt_tunables* tunables) {
+  if (dtype != LT_DTYPE_BF16 || T <= 0 || N <= 0 || !scan_knn_supported(D) || topk <= 0 || topk > N || topk > LT_MAX_TOPK) return 0;
+  return make_layout(true, T, N, topk, N - 1, resolve_tunables(tunables)).total;
+}
+
+int lt_knn_scores(int dtype, const void* q, const void* x, int T, int N, int D, int row_begin, int row_end, float* out_scores,
+                  void* stream_) {
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  int rc = knn_check(dtype, q, x, T, N, D);
+  if (rc != LT_OK) return rc;
+  if (out_scores == nullptr || row_begin < 0 || row_end > T || row_begin > row_end) return LT_ERR_INVALID_ARG;
+  if (row_begin == row_end) return LT_OK;
+  Control* ctl = nullptr;
+  LT_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&ctl), g_scores_ctl));
+  const int grid = sm_count();
+  KnnScanParams p{};
+  p.T = T;
+  p.row_begin = row_begin;
+  p.row_end = row_end;
+  p.n_keys = N;
+  p.D = D;
+  p.seg_tiles = knn_seg_tiles(resolve_tunables(nullptr), N, grid);
+  p.dump = out_scores;
+  p.dump_ld = N;
+  p.ctl = ctl;
+  LT_LAUNCH(launch_scan_knn(kModeDump, q, T, x, N, D, p, grid, stream));
+  return LT_OK;
+}
+
+int lt_knn_topk(int dtype, const void* q, const void* x, int T, int N, int D, int topk, int32_t* out_idx, float* out_score,
+                void* workspace, size_t workspace_bytes, const lt_tunables* tunables, void* stream_) {
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  int rc = knn_check(dtype, q, x, T, N, D);
+  if (rc != LT_OK) return rc;
+  if (out_idx == nullptr || topk <= 0 || topk > N || topk > LT_MAX_TOPK) return LT_ERR_INVALID_ARG;
+  const Tun tun = resolve_tunables(tunables);
+  const Layout L = make_layout(true, T, N, topk, N - 1, tun);  // every query sees the whole corpus
+  if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) != 0 || workspace_bytes < L.total)
+    return LT_ERR_WORKSPACE;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  Control* ctl = reinterpret_cast<Control*>(ws + L.ctl);
+  LT_CUDA(cudaMemsetAsync(ws, 0, L.zero_end, stream));
+  const int grid = tun.grid > 0 ? tun.grid : sm_count();
+  float* smin = reinterpret_cast<float*>(ws + L.smin);
+  float* width = reinterpret_cast<float*>(ws + L.width);
+  float* thr = reinterpret_cast<float*>(ws + L.thr);
+  unsigned int* tail = reinterpret_cast<unsigned int*>(ws + L.tail);
+  unsigned int* hist = reinterpret_cast<unsigned int*>(ws + L.hist);
+  unsigned char* row_flag = ws + L.row_flag;
+  unsigned int* block_flag = reinterpret_cast<unsigned int*>(ws + L.block_flag);
+  int* fb_list = reinterpret_cast<int*>(ws + L.fb_list);
+  float* sample = reinterpret_cast<float*>(ws + L.sample);
+  uint2* cand = reinterpret_cast<uint2*>(ws + L.cand);
+  float* scratch = reinterpret_cast<float*>(ws + L.scratch);
+
+  // 1. sample phase (paper Sec. 3.2 "Sampling": "for k-NN search ... random sampling suffices"): a strided
+  //    view of the corpus, scored by the same tensor-core kernel
+  mark_phase(0, stream);
+  if (L.n_sample > 0) {
+    KnnScanParams p{};
+    p.T = T;
+    p.row_begin = 0;
+    p.row_end = T;
+    p.n_keys = L.n_sample;
+    p.D = D;
+    p.seg_tiles = knn_seg_tiles(tun, L.n_sample, grid);
+    p.dump = sample;
+    p.dump_ld = L.n_sample;
+    p.ctl = ctl;
+    LT_LAUNCH(launch_scan_knn(kModeDump, q, T, x, L.n_sample, static_cast<long long>(L.sample_stride) * D, p, grid, stream));
+  }
+  mark_phase(1, stream);
+  LT_LAUNCH(launch_sample_stats(sample, T, L.n_sample, L.sample_rank, smin, width, thr, stream));
+  mark_phase(2, stream);
+
+  // 2. fused scan: one pass over the corpus
+  {
+    KnnScanParams p{};
+    p.T = T;
+    p.row_begin = 0;
+    p.row_end = T;
+    p.n_keys = N;
+    p.D = D;
+    p.seg_tiles = knn_seg_tiles(tun, N, grid);
+    p.topk = topk;
+    p.thr = thr;
+    p.smin = smin;
+    p.width = width;
+    p.tail = tail;
+    p.hist = hist;
+    p.cand = cand;
+    p.cap = L.cap;
+    p.ctl = ctl;
+    LT_LAUNCH(launch_scan_knn(kModeFilter, q, T, x, N, D, p, grid, stream));
+  }
+
+  // 3. final select; rows it cannot finish exactly are flagged
+  mark_phase(3, stream);
+  {
+    FinalSelectParams p{};
+    p.tail = tail;
+    p.hist = hist;
+    p.cand = cand;
+    p.smin = smin;
+    p.width = width;
+    p.cap = L.cap;
+    p.T = T;
+    p.N = N;
+    p.topk = topk;
+    p.causal_offset = N;  // no causal mask
+    p.out_idx = out_idx;
+    p.out_score = out_score;
+    p.row_flag = row_flag;
+    p.block_flag = block_flag;
+    p.fb_list = fb_list;
+    p.ctl = ctl;
+    LT_LAUNCH(launch_final_select(p, stream));
+  }
+
+  // 4. exact fallback, one block of 8 rows at a time: dense scores of the block (a launch whose block nobody
+  //    flagged returns at once), then the full-row select for the flagged rows
+  mark_phase(4, stream);
+  for (int b = 0; b < L.n_blocks; ++b) {
+    const int r0 = b * kRowsPerBlock;
+    const int r1 = r0 + kRowsPerBlock < T ? r0 + kRowsPerBlock : T;
+    KnnScanParams p{};
+    p.T = T;
+    p.row_begin = r0;
+    p.row_end = r1;
+    p.n_keys = N;
+    p.D = D;
+    p.seg_tiles = knn_seg_tiles(tun, N, grid);
+    p.dump = scratch;
+    p.dump_ld = N;
+    p.fb_flag = block_flag;
+    p.ctl = ctl;
+    LT_LAUNCH(launch_scan_knn(kModeDump, q, T, x, N, D, p, grid, stream));
+    SelectRowsParams sp{};
+    sp.scores = scratch;
+    sp.ld = N;
+    sp.n_blocks = r1 - r0;
+    sp.row_begin = r0;
+    sp.T = T;
+    sp.N = N;
+    sp.topk = topk;
+    sp.causal_offset = N;
+    sp.out_idx = out_idx;
+    sp.out_score = out_score;
+    sp.row_flag = row_flag;
+    sp.ctl = ctl;
+    LT_LAUNCH(launch_select_rows(sp, stream));
+  }
+  mark_phase(5, stream);
+  return LT_OK;
+}
+
 int lt_unfused_topk(int dtype, const void* q, const float* w, const void* k, const float* k_scale, int T, int N, int H, int D,
                     int topk, int causal_offset, int32_t* out_idx, float* out_score, float* score_buf, size_t score_buf_bytes,
                     int path, void* stream_) {

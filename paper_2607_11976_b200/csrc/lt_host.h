@@ -51,6 +51,34 @@ bool scan_mma_supported(int dtype, int H, int D);
 cudaError_t launch_scan_mma(int dtype, int mode, const void* q, int T, const void* k, long long n_keys_view,
                             long long key_pitch_elems, const ScanParams& p, int grid, cudaStream_t stream);
 
+// ---- lt_scan_knn.cu -------------------------------------------------------------------------
+// Parameters of the tensor-core scan of the k-NN (inner-product) variant: bf16 queries [T][D], corpus view of
+// n_keys rows, every row sees every key.
+struct KnnScanParams {
+  int T;                   // rows of q
+  int row_begin, row_end;  // query rows handled by this launch
+  int n_keys;              // corpus vectors in the view
+  int D;                   // multiple of 64, at most 768
+  int seg_tiles;           // corpus tiles (128 vectors) per work item
+  int topk;
+  // filter mode
+  float* thr;              // [T] gate: lower edge of the row's threshold bin
+  const float* smin;       // [T]
+  const float* width;      // [T]
+  unsigned int* tail;      // [T]
+  unsigned int* hist;      // [T][kBins]
+  uint2* cand;             // [T][cap]
+  int cap;
+  // dump mode
+  float* dump;             // dense scores, row (t - row_begin)
+  long long dump_ld;
+  const unsigned int* fb_flag;  // fallback rounds: flag per block of 8 rows; the launch is a no-op if its block's flag is 0
+  Control* ctl;
+};
+bool scan_knn_supported(int D);
+cudaError_t launch_scan_knn(int mode, const void* q, int T, const void* x, long long n_keys_view, long long key_pitch_elems,
+                            const KnnScanParams& p, int grid, cudaStream_t stream);
+
 // ---- lt_select.cu ---------------------------------------------------------------------------
 // Generic SIMT scoring (any H, D, dtype): dense scores of rows [row_begin, row_end), -inf where masked.
 cudaError_t launch_simt_scores(int dtype, const void* q, const float* w, const void* k, const float* k_scale, int T, int N,

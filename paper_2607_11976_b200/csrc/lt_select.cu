@@ -263,6 +263,7 @@ __global__ void __launch_bounds__(kSelThreads) select_rows_kernel(const SelectRo
     if (t >= p.T || !p.row_flag[t]) return;
   } else {
     t = p.row_begin + blockIdx.x;
+    if (p.row_flag != nullptr && !p.row_flag[t]) return;  // only flagged rows are redone
   }
   const float* row = p.scores + static_cast<size_t>(blockIdx.x) * p.ld;
   const int vis = visible_keys(t, p.N, p.causal_offset);
