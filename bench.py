@@ -235,6 +235,148 @@ def time_aux_ops(torch, lt, out_idx, inp, hbm_gbs, peak_kind, reps=5):
     return out
 
 
+def run_knn(args, rank: int, local_rank: int, world: int):
+    """k-NN (inner-product) variant: one step = exact top-k of a batch of queries over the whole corpus."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_2607_11976_b200 import binding as lt
+    from paper_2607_11976_b200 import build as lt_build
+    from workloads import make_knn
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    args.warmup = max(args.warmup, 3)
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        lt_build.build()
+    if world > 1:
+        dist.barrier()
+    lt.load()
+    inp = make_knn(args.workload, N=args.knn_corpus or None)
+    pairs = inp.valid_pairs()
+    q = torch.from_numpy(inp.q.view("int16")).cuda().view(torch.bfloat16)
+    x = torch.from_numpy(inp.x.view("int16")).cuda().view(torch.bfloat16)
+    out_idx = torch.empty((inp.T, inp.topk), dtype=torch.int32, device="cuda")
+    out_score = torch.empty((inp.T, inp.topk), dtype=torch.float32, device="cuda")
+    ws = torch.empty(lt.lt_knn_topk_workspace_bytes(inp.T, inp.N, inp.D, inp.topk), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step():
+        lt.lt_knn_topk(q, x, inp.topk, out_idx, out_score, ws)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    lt.lt_set_profiling(True)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    for _ in range(args.warmup):
+        step()
+    # a step lasts well under the clock sampler's period: keep the same load up for half a second (untimed) so
+    # that the sampled clocks and throttle reasons describe the state the timed steps run in
+    t_load = time.perf_counter()
+    while time.perf_counter() - t_load < 0.5:
+        step()
+        torch.cuda.synchronize()
+    status = lt.lt_read_status(ws)
+    if status[0] & lt.LT_STATUS_TIMEOUT:
+        raise SystemExit("device-side wait timed out; results invalid")
+    barrier()
+    launches0 = lt.lt_launch_count()
+    step_ms, phase_ms = [], []
+    for _ in range(args.steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        step()
+        e1.record(stream)
+        e1.synchronize()
+        step_ms.append(e0.elapsed_time(e1))
+        phase_ms.append(lt.lt_read_phase_ms())
+    launches = lt.lt_launch_count() - launches0
+    barrier()
+    clocks = sampler.stop()
+    total_ms = max_over_ranks(sum(step_ms), world, "cuda")
+    ms_per_step = total_ms / args.steps
+    value = aggregate_throughput(pairs, args.steps, total_ms, world)
+    status = lt.lt_read_status(ws)
+
+    host = [q.cpu().pin_memory(), x.cpu().pin_memory()]
+    h_idx = torch.empty_like(out_idx, device="cpu").pin_memory()
+    h_score = torch.empty_like(out_score, device="cpu").pin_memory()
+
+    def e2e_step():
+        q.copy_(host[0], non_blocking=True)
+        x.copy_(host[1], non_blocking=True)
+        step()
+        h_idx.copy_(out_idx, non_blocking=True)
+        h_score.copy_(out_score, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e2e_steps = min(args.steps, 3)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    e1.synchronize()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peaks, peak_kind = load_peaks()
+    scan_ms = statistics.mean(p[2] for p in phase_ms)
+    # algorithmic bytes of the scan: the corpus once per block of 64 queries, the queries, the survivors
+    n_qblocks = -(-inp.T // 64)
+    alg_bytes = n_qblocks * inp.N * inp.D * 2 + inp.T * inp.D * 2 + status[3] * 8
+    achieved = alg_bytes / (scan_ms * 1e-3) / 1e9
+    names = ["sample_scan", "sample_stats", "fused_scan", "final_select", "fallback"]
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": args.workload, "T": inp.T, "N": inp.N, "D": inp.D, "topk": inp.topk, "valid_pairs": pairs,
+                   "parallelism": f"replicas x{world}", "l2": "inputs larger than L2 (corpus streamed once per step)",
+                   "workspace_bytes": int(ws.numel())},
+        "clocks": clocks,
+        "e2e": {"value": aggregate_throughput(pairs, e2e_steps, e2e_ms, world), "unit": UNIT,
+                "h2d_bytes_per_step": sum(t.numel() * t.element_size() for t in host),
+                "d2h_bytes_per_step": h_idx.numel() * 4 + h_score.numel() * 4, "ms_per_step": e2e_ms / e2e_steps},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "kernel": "knn_scan_kernel (fused score + filter)", "achieved": achieved,
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",
+                     "kernel_ms": scan_ms, "algorithmic_bytes": alg_bytes, "traffic": None},
+        "phases_ms": {n: statistics.mean(p[i] for p in phase_ms) for i, n in enumerate(names)},
+        "status": {"bits": status[0], "fallback_rows": status[1], "max_survivors_per_row": status[2],
+                   "mean_survivors_per_row": status[3] / inp.T, "overflow_rows": status[4]},
+    }
+    if not args.no_cpu_baseline and world == 1:
+        from oracle import knn_topk
+
+        np.matmul(np.ones((64, 64)), np.ones((64, 64)))
+        t0 = time.perf_counter()
+        rows_done = 0
+        for r in range(0, inp.T, 4):
+            knn_topk(inp.q, inp.x, inp.topk, rows=list(range(r, min(inp.T, r + 4))))
+            rows_done += min(inp.T, r + 4) - r
+            if time.perf_counter() - t0 > args.cpu_budget:
+                break
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": rows_done * inp.N / dt, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                                "sample": f"{rows_done} query rows x the whole corpus ({rows_done * inp.N} pairs, {dt:.1f} s)"}
+    else:
+        line["cpu_baseline"] = None
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -250,6 +392,7 @@ def main():
     ap.add_argument("--aux", action="store_true",
                     help="also time the auxiliary integer ops on this step's top-k result: lt_topk_frequent and "
                          "lt_dsa_union_mask (group 64); adds an 'aux' object to the JSON line")
+    ap.add_argument("--knn-corpus", type=int, default=0, help="k-NN workloads: corpus size (default: the workload's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-unfused", action="store_true")
     ap.add_argument("--unfused-budget-mb", type=int, default=2048, help="score-matrix budget of the unfused GPU baseline")
@@ -261,6 +404,10 @@ def main():
 
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+
+    if args.workload.startswith("knn"):
+        run_knn(args, rank, local_rank, world)
         return
 
     import torch

@@ -37,13 +37,21 @@ constexpr int kQB = 64;                      // queries per block = UMMA N
 constexpr int kSliceElems = 64;              // bf16 elements in a 128-byte row piece
 constexpr int kQSliceBytes = kQB * 128;      // 8 KB: 64 query rows x 128 bytes
 constexpr int kXSliceBytes = kTileKeys * 128;  // 16 KB: 128 corpus rows x 128 bytes
-constexpr int kKnnStages = 6;
+#ifndef LT_KNN_STAGES
+#define LT_KNN_STAGES 6
+#endif
+constexpr int kKnnStages = LT_KNN_STAGES;
+#ifndef LT_KNN_PF
+#define LT_KNN_PF 0
+#endif
+constexpr int kKnnPrefetchTiles = LT_KNN_PF;         // corpus tiles requested into L2 ahead of the shared-memory ring
 constexpr int kKnnMaxSlices = 12;            // D <= 768
 constexpr int kAccBufs = 4;                  // TMEM accumulators of 64 columns
 constexpr int kKnnTmemCols = kAccBufs * kQB;  // 256
 constexpr int kKnnFirstEpi = 3;
 constexpr int kKnnEpiWarps = 8;
 constexpr int kKnnThreads = (kKnnFirstEpi + kKnnEpiWarps) * 32;
+constexpr int kKnnStageLen = 128;            // entries of one warp's staging list
 
 struct KnnTail {
   float thr[kQB];
@@ -60,6 +68,7 @@ struct KnnTail {
   int abort_flag;
   int epi_abort;
   int done_seq;
+  uint4 stage[kKnnEpiWarps][kKnnStageLen];  // per warp: (score bits, corpus index, query row, -) of survivors
 };
 
 constexpr int knn_smem_bytes(int n_slices) { return 1024 + n_slices * kQSliceBytes + kKnnStages * kXSliceBytes + static_cast<int>(sizeof(KnnTail)); }
@@ -81,19 +90,65 @@ __device__ __forceinline__ bool knn_item(const KnnScanParams& p, int qb_lo, int 
   return it.tile_lo < it.tile_hi;
 }
 
-// Survivors of one ballot go straight to the query's candidate buffer: one tail atomic for the warp, then
-// each passing lane stores its entry and counts it in the query's histogram (fire-and-forget).  Entries
-// beyond the capacity are dropped but still counted: the tail then exceeds the capacity, which flags the row.
-__device__ __forceinline__ void knn_append(bool pass, uint32_t ballot, float score, int s, const KnnScanParams& p, int t, int lane,
-                                           float smin, float width, float inv_width) {
-  uint32_t base = 0;
-  if (lane == 0) base = atomicAdd(p.tail + t, static_cast<uint32_t>(__popc(ballot)));
-  base = __shfl_sync(0xffffffffu, base, 0);
-  if (pass) {
-    const uint32_t pos = base + __popc(ballot & ((1u << lane) - 1u));
-    if (pos < static_cast<uint32_t>(p.cap)) p.cand[static_cast<size_t>(t) * p.cap + pos] = make_uint2(__float_as_uint(score), static_cast<uint32_t>(s));
-    atomicAdd(p.hist + static_cast<size_t>(t) * kBins + bin_of(score, smin, width, inv_width), 1u);
+// Gate of 32 queries against one corpus vector per lane: bit q of the result = score[q] >= thr[q].
+// The thresholds are read as eight 16-byte volatile loads (they move while the scan runs).
+__device__ __forceinline__ uint32_t knn_gate32(const uint32_t (&v)[32], const float* thr, bool in_range) {
+  uint32_t m = 0;
+#pragma unroll
+  for (int j = 0; j < 32; j += 4) {
+    float t0, t1, t2, t3;
+    asm volatile("ld.volatile.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(t0), "=f"(t1), "=f"(t2), "=f"(t3) : "r"(smem_u32(thr + j)));
+    m |= (__uint_as_float(v[j + 0]) >= t0 ? 1u : 0u) << (j + 0);
+    m |= (__uint_as_float(v[j + 1]) >= t1 ? 1u : 0u) << (j + 1);
+    m |= (__uint_as_float(v[j + 2]) >= t2 ? 1u : 0u) << (j + 2);
+    m |= (__uint_as_float(v[j + 3]) >= t3 ? 1u : 0u) << (j + 3);
   }
+  return in_range ? m : 0u;
+}
+
+// Survivors go to one staging list per warp in shared memory, (score bits, corpus index, query row, -), for
+// all 64 queries together: appending costs a ballot and a shared-memory store, nothing waits for global
+// memory.  A list that may not hold the next ballot is flushed: every lane reserves a slot in its entry's
+// candidate buffer with its own atomic (all of them in flight together: one round trip per 32 entries), stores
+// the entry and counts it in the query's histogram.  Entries beyond the capacity are dropped but still counted
+// (the tail then exceeds the capacity, which flags the row).  Paper Sec. 3.2 "Filtering": "a list in warp-local
+// shared memory, flushed in batches".
+__device__ __noinline__ void knn_flush(const uint4* list, int count, const KnnScanParams& p, int t0, const float* smin,
+                                       const float* width, const float* inv_width) {
+  const int lane = threadIdx.x & 31;
+  __syncwarp();
+  for (int i = lane; i < count; i += 32) {
+    const uint4 e = list[i];
+    const int t = static_cast<int>(e.z);
+    const uint32_t pos = atomicAdd(p.tail + t, 1u);
+    if (pos < static_cast<uint32_t>(p.cap)) p.cand[static_cast<size_t>(t) * p.cap + pos] = make_uint2(e.x, e.y);
+    const int r = t - t0;
+    atomicAdd(p.hist + static_cast<size_t>(t) * kBins + bin_of(__uint_as_float(e.x), smin[r], width[r], inv_width[r]), 1u);
+  }
+  __syncwarp();
+}
+
+// Appends the survivors of 32 queries (bit q of `mine`: this lane's vector survives query q; bit q of `any`: some
+// lane's does).  Returns the new list length.
+__device__ __forceinline__ int knn_stage32(uint32_t any, uint32_t mine, const uint32_t (&v)[32], int s, int t_first, int lane,
+                                           uint4* list, int count, const KnnScanParams& p, int t0, const float* smin,
+                                           const float* width, const float* inv_width) {
+#pragma unroll
+  for (int q = 0; q < 32; ++q) {
+    if ((any >> q) & 1u) {
+      const bool pass = (mine >> q) & 1u;
+      const uint32_t bal = __ballot_sync(0xffffffffu, pass);
+      if (count + 32 > kKnnStageLen) {
+        knn_flush(list, count, p, t0, smin, width, inv_width);
+        count = 0;
+      }
+      // + 0 turns -0 into +0, so that the bit order of the scores is their value order
+      if (pass) list[count + __popc(bal & ((1u << lane) - 1u))] =
+          make_uint4(__float_as_uint(__fadd_rn(__uint_as_float(v[q]), 0.f)), static_cast<uint32_t>(s), static_cast<uint32_t>(t_first + q), 0u);
+      count += __popc(bal);
+    }
+  }
+  return count;
 }
 
 template <int kMode>
@@ -173,6 +228,9 @@ knn_scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (!ok) break;
             mbar_arrive_expect_tx(smem_u32(&st->bar_full[stage]), kXSliceBytes);
             tma_load_2d(x_base + stage * kXSliceBytes, &tm_x, sl * kSliceElems, tile * kTileKeys, smem_u32(&st->bar_full[stage]));
+            // the ring holds 112 KB per SM, less than HBM's bandwidth-delay product needs: ask L2 for the same
+            // slice of a later tile now (no completion to wait for; rows past the corpus are simply not fetched)
+            if (kKnnPrefetchTiles > 0 && tile + kKnnPrefetchTiles < it.tile_hi) tma_prefetch_2d(&tm_x, sl * kSliceElems, (tile + kKnnPrefetchTiles) * kTileKeys);
             if (++stage == kKnnStages) {
               stage = 0;
               phase ^= 1;
@@ -237,13 +295,31 @@ knn_scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const int key_in_tile = quarter * 32 + lane;
       const uint32_t tlane = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
       uint32_t seq = 0;  // tiles this CTA has gone through (same count as the UMMA warp's)
-      int item_seq = 0;
+      // An "epoch" is a run of consecutive work items on the same query block: the per-query state in shared
+      // memory is loaded, and the warps meet, only when the block changes (with one block of 64 queries: once).
+      int item_seq = 0;  // epoch number
+      int cur_qb = -1;
+      int n_staged = 0;   // entries in this warp's staging list (warp-uniform)
+      bool dead = false;  // a wait gave up: skip the remaining work, keep meeting the barriers
       for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
         KnnItem it;
         if (!knn_item(p, qb_lo, n_qb, item, it)) continue;
-        ++item_seq;
         const int t0 = it.qb * kQB;
-        named_bar_sync(1, n_sync);  // A: everybody is done with the previous item's shared state
+        if (it.qb == cur_qb) {
+          if (is_refresh) continue;  // the refresh warp served the whole epoch when it began
+        } else {
+        if (cur_qb >= 0 && !is_refresh) {
+          // the previous epoch is over when both sets are through: tell the refresh warp
+          if (kMode == kModeFilter && n_staged > 0) {
+            knn_flush(st->stage[ew], n_staged, p, cur_qb * kQB, st->smin, st->width, st->inv_width);
+            n_staged = 0;
+          }
+          named_bar_sync(2, kEpiThreads);
+          if (warp == kKnnFirstEpi && lane == 0) *reinterpret_cast<volatile int*>(&st->done_seq) = item_seq;
+        }
+        ++item_seq;
+        cur_qb = it.qb;
+        named_bar_sync(1, n_sync);  // A: everybody is done with the previous epoch's shared state
         if (!is_refresh) {
           if (e < kQB && kMode == kModeFilter) {
             const int t = t0 + e;
@@ -261,11 +337,15 @@ knn_scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (is_refresh) {
           // ---- paper Sec. 3.2 "Threshold Refresh": per query, walk the histogram from the top bin down until
           // the cumulative count reaches k and publish that bin's lower edge by plain store
+          // A pass over 64 histograms takes tens of microseconds, a work item about as long: the end of the
+          // item is checked before every row so that the epilogue warps never wait for this warp.
           unsigned int sleep_ns = 2000;
-          while (true) {
-            for (int r = 0; r < kQB; ++r) {
+          bool done = false;
+          while (!done) {
+            for (int r = 0; r < kQB && !done; ++r) {
               const int t = t0 + r;
-              if (t < p.row_begin || t >= p.row_end) continue;
+              done = *reinterpret_cast<volatile int*>(&st->done_seq) >= item_seq || *abort_flag;
+              if (done || t < p.row_begin || t >= p.row_end) continue;
               const uint4* hp = reinterpret_cast<const uint4*>(p.hist + static_cast<size_t>(t) * kBins + lane * 8);
               const uint4 h0 = __ldcg(hp), h1 = __ldcg(hp + 1);
               const uint32_t c[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
@@ -302,19 +382,18 @@ knn_scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
               }
             }
-            bool done = false;
             for (unsigned int slept = 0; slept < sleep_ns && !done; slept += 1000) {
               __nanosleep(1000);
               done = *reinterpret_cast<volatile int*>(&st->done_seq) >= item_seq || *abort_flag;
             }
-            if (done) break;
             if (sleep_ns < 32000) sleep_ns += sleep_ns >> 1;
           }
           continue;
         }
+        }  // epoch change
 
         // ---- epilogue proper: this warp drains the tiles of its set for its 32 corpus vectors
-        bool ok = true;
+        bool ok = !dead;
         for (int tile = it.tile_lo; tile < it.tile_hi && ok; ++tile, ++seq) {
           if ((seq & 1u) != set) continue;
           const uint32_t buf = seq & (kAccBufs - 1);
@@ -330,23 +409,30 @@ knn_scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           if (lane == 0) mbar_arrive(smem_u32(&st->bar_acc_empty[buf]));
           if (!ok) break;
           const bool in_range = s < p.n_keys;
+          if (kMode == kModeDump) {
 #pragma unroll
-          for (int qq = 0; qq < kQB; ++qq) {
-            // + 0 turns -0 into +0, so that the bit order of the scores is their value order
-            const float score = __fadd_rn(__uint_as_float(qq < 32 ? va[qq & 31] : vb[qq & 31]), 0.f);
-            const int t = t0 + qq;
-            if (kMode == kModeDump) {
+            for (int qq = 0; qq < kQB; ++qq) {
+              // + 0 turns -0 into +0, so that the bit order of the scores is their value order
+              const float score = __fadd_rn(__uint_as_float(qq < 32 ? va[qq & 31] : vb[qq & 31]), 0.f);
+              const int t = t0 + qq;
               if (in_range && t >= p.row_begin && t < p.row_end) p.dump[static_cast<size_t>(t - p.row_begin) * p.dump_ld + s] = score;
-            } else {
-              // ---- paper Sec. 3.2 "Filtering": a compare per score; rows outside the launch have thr = +inf
-              const float thr = *reinterpret_cast<volatile float*>(&st->thr[qq]);
-              const bool pass = in_range && (score >= thr);
-              const uint32_t ballot = __ballot_sync(0xffffffffu, pass);
-              if (ballot != 0) knn_append(pass, ballot, score, s, p, t, lane, st->smin[qq], st->width[qq], st->inv_width[qq]);
             }
+          } else {
+            // ---- paper Sec. 3.2 "Filtering": a compare per score (rows outside the launch have thr = +inf;
+            // -0 and +0 compare alike, so the raw accumulator is gated), then the few (query, warp) pairs
+            // with a survivor are written out
+            const uint32_t ma = knn_gate32(va, st->thr, in_range);
+            const uint32_t mb = knn_gate32(vb, st->thr + 32, in_range);
+            const uint32_t any_a = __reduce_or_sync(0xffffffffu, ma);
+            const uint32_t any_b = __reduce_or_sync(0xffffffffu, mb);
+            if (any_a != 0u) n_staged = knn_stage32(any_a, ma, va, s, t0, lane, st->stage[ew], n_staged, p, t0, st->smin, st->width, st->inv_width);
+            if (any_b != 0u) n_staged = knn_stage32(any_b, mb, vb, s, t0 + 32, lane, st->stage[ew], n_staged, p, t0, st->smin, st->width, st->inv_width);
           }
         }
-        // the item is over when both sets are through
+        if (!ok) dead = true;
+      }
+      if (cur_qb >= 0 && !is_refresh) {
+        if (kMode == kModeFilter && n_staged > 0) knn_flush(st->stage[ew], n_staged, p, cur_qb * kQB, st->smin, st->width, st->inv_width);
         named_bar_sync(2, kEpiThreads);
         if (warp == kKnnFirstEpi && lane == 0) *reinterpret_cast<volatile int*>(&st->done_seq) = item_seq;
       }
