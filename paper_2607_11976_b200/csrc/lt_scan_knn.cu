@@ -37,14 +37,7 @@ constexpr int kQB = 64;                      // queries per block = UMMA N
 constexpr int kSliceElems = 64;              // bf16 elements in a 128-byte row piece
 constexpr int kQSliceBytes = kQB * 128;      // 8 KB: 64 query rows x 128 bytes
 constexpr int kXSliceBytes = kTileKeys * 128;  // 16 KB: 128 corpus rows x 128 bytes
-#ifndef LT_KNN_STAGES
-#define LT_KNN_STAGES 6
-#endif
-constexpr int kKnnStages = LT_KNN_STAGES;
-#ifndef LT_KNN_PF
-#define LT_KNN_PF 0
-#endif
-constexpr int kKnnPrefetchTiles = LT_KNN_PF;         // corpus tiles requested into L2 ahead of the shared-memory ring
+constexpr int kKnnStages = 6;                // 16 KB K-slices in flight per SM (a seventh, or L2 prefetches ahead, gained nothing)
 constexpr int kKnnMaxSlices = 12;            // D <= 768
 constexpr int kAccBufs = 4;                  // TMEM accumulators of 64 columns
 constexpr int kKnnTmemCols = kAccBufs * kQB;  // 256
@@ -228,9 +221,6 @@ knn_scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (!ok) break;
             mbar_arrive_expect_tx(smem_u32(&st->bar_full[stage]), kXSliceBytes);
             tma_load_2d(x_base + stage * kXSliceBytes, &tm_x, sl * kSliceElems, tile * kTileKeys, smem_u32(&st->bar_full[stage]));
-            // the ring holds 112 KB per SM, less than HBM's bandwidth-delay product needs: ask L2 for the same
-            // slice of a later tile now (no completion to wait for; rows past the corpus are simply not fetched)
-            if (kKnnPrefetchTiles > 0 && tile + kKnnPrefetchTiles < it.tile_hi) tma_prefetch_2d(&tm_x, sl * kSliceElems, (tile + kKnnPrefetchTiles) * kTileKeys);
             if (++stage == kKnnStages) {
               stage = 0;
               phase ^= 1;

@@ -103,3 +103,16 @@ def test_bad_arguments():
         lt.lt_knn_topk(q, x, 8, out, None, ws[:512])
     assert e.value.code == -3
     assert lt.lt_knn_topk_workspace_bytes(4, 500, 100, 8) == 0
+
+
+def test_full_size_benchmark_shape():
+    """The shape bench.py times (64 queries x 1,048,576 vectors x 768, k = 1024, default tunables): every row
+    against the oracle's index and score rules, and bit-exactly against the library's own dumped scores."""
+    inp = make_knn()
+    idx, score, st = gpu_topk(inp)
+    assert st[0] == 0 and st[1] == 0, st
+    srt = np.sort(idx, axis=1)
+    assert idx.min() >= 0 and idx.max() < inp.N and np.all(srt[:, 1:] != srt[:, :-1])
+    assert np.all(np.diff(score.astype(np.float64), axis=1) <= 0)
+    dumped = np.concatenate([gpu_scores(inp, r, r + 16) for r in range(0, inp.T, 16)])
+    check(inp, idx, score, list(range(inp.T)), dumped)
