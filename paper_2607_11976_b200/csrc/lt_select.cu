@@ -135,6 +135,89 @@ __device__ __forceinline__ void sort_and_write(uint64_t* sel, int count, int top
 }
 
 // ---------------------------------------------------------------------------------------------
+// Keeps the `keep` largest of the `count` distinct 64-bit keys in sel[0 .. count), compacted to sel[0 .. keep)
+// in any order.  MSB radix select, 8 bits per pass, histogram in shared memory (hist: 256 counters, scratch: one
+// counter); the digit of each pass is found by a warp suffix scan.  Called by every thread of the CTA.
+// ---------------------------------------------------------------------------------------------
+constexpr int kKeepPerThread = 8;  // keys a thread holds in registers per compaction slab
+__device__ __forceinline__ void keep_top_keys(uint64_t* sel, int count, int keep, unsigned int* hist, unsigned int* scratch) {
+  __shared__ uint64_t s_prefix64;
+  __shared__ unsigned int s_need;
+  const int tid = threadIdx.x, lane = tid & 31, nthreads = blockDim.x;
+  if (tid == 0) {
+    s_prefix64 = 0;
+    s_need = static_cast<unsigned int>(keep);
+  }
+  uint64_t mask = 0;
+  for (int pass = 0; pass < 8; ++pass) {
+    const int shift = 56 - 8 * pass;
+    if (tid < 256) hist[tid] = 0;
+    __syncthreads();
+    const uint64_t prefix = s_prefix64;
+    for (int i = tid; i < count; i += nthreads) {
+      const uint64_t key = sel[i];
+      if ((key & mask) == prefix) atomicAdd(&hist[static_cast<unsigned int>(key >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (tid < 32) {
+      // suffix sums over the 256 digits, 8 per lane: the digit where the count from the top reaches `need`
+      unsigned int c[8], mine = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        c[j] = hist[lane * 8 + j];
+        mine += c[j];
+      }
+      unsigned int incl = mine;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const unsigned int o = __shfl_down_sync(0xffffffffu, incl, d);
+        if (lane + d < 32) incl += o;
+      }
+      const unsigned int above = incl - mine, need = s_need;
+      if (above < need && incl >= need) {  // exactly one lane
+        unsigned int cum = above;
+        for (int j = 7; j >= 0; --j) {
+          if (cum + c[j] >= need) {
+            s_prefix64 = prefix | (static_cast<uint64_t>(lane * 8 + j) << shift);
+            s_need = need - cum;
+            break;
+          }
+          cum += c[j];
+        }
+      }
+    }
+    mask |= 0xffull << shift;
+    __syncthreads();
+  }
+  const uint64_t kth = s_prefix64;  // the keep-th largest key itself
+  // compaction in place, a slab of kKeepPerThread * nthreads keys at a time: every thread pulls its keys of
+  // the slab into registers, then the kept ones are written from the front (never past what has been read)
+  if (tid == 0) *scratch = 0;
+  for (int slab = 0; slab < count; slab += kKeepPerThread * nthreads) {
+    uint64_t mine[kKeepPerThread];
+#pragma unroll
+    for (int j = 0; j < kKeepPerThread; ++j) {
+      const int i = slab + j * nthreads + tid;
+      mine[j] = i < count ? sel[i] : 0ull;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < kKeepPerThread; ++j) {
+      const int i = slab + j * nthreads + tid;
+      const bool take = i < count && mine[j] >= kth;
+      const unsigned int ballot = __ballot_sync(0xffffffffu, take);
+      if (ballot != 0) {
+        unsigned int base = 0;
+        if (lane == 0) base = atomicAdd(scratch, static_cast<unsigned int>(__popc(ballot)));
+        base = __shfl_sync(0xffffffffu, base, 0);
+        if (take) sel[base + __popc(ballot & ((1u << lane) - 1u))] = mine[j];
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // final select over one row's candidate buffer (paper Sec. 3.2 "Top-k Selection"): the final
 // threshold bin is the highest bin whose cumulative count from the top reaches k; every candidate
 // at or above its lower edge is pulled into shared memory (the bins above hold fewer than k of
@@ -230,7 +313,15 @@ __global__ void __launch_bounds__(kFinalThreads) final_select_kernel(const Final
     // count < kk cannot happen for an exact filter; treating it as "redo" keeps the result exact regardless
     if (count > static_cast<unsigned int>(sel_cap) || count < static_cast<unsigned int>(kk)) redo = true;
     if (!redo) {
-      sort_and_write(sel, static_cast<int>(count), p.topk, p.out_idx + static_cast<size_t>(t) * p.topk,
+      int n_keep = static_cast<int>(count);
+      if (n_keep > kk && kk > 0) {
+        // More candidates than outputs (the threshold bin is included whole).  The packed keys are distinct
+        // (the index is part of them), so the kk-th largest key is unique: find it by an 8-pass radix select
+        // in shared memory and keep exactly the keys at or above it, which halves the sort that follows.
+        keep_top_keys(sel, n_keep, kk, hist, &s_count);
+        n_keep = kk;
+      }
+      sort_and_write(sel, n_keep, p.topk, p.out_idx + static_cast<size_t>(t) * p.topk,
                      p.out_score ? p.out_score + static_cast<size_t>(t) * p.topk : nullptr);
       return;
     }
