@@ -52,13 +52,17 @@ constexpr size_t kGenericScratchBudget = size_t(256) << 20;   // dense scores ke
 
 struct Tun {
   int path, cap_mult, sample_mult, segment_tiles, grid, sample_rank;
+  bool sample_mult_given;
 };
 Tun resolve_tunables(const lt_tunables* t) {
-  Tun r{LT_PATH_AUTO, 12, 3, 0, 0, 0};
+  Tun r{LT_PATH_AUTO, 12, 3, 0, 0, 0, false};
   if (t != nullptr) {
     r.path = t->path;
     if (t->cap_mult > 0) r.cap_mult = t->cap_mult;
-    if (t->sample_mult > 0) r.sample_mult = t->sample_mult;
+    if (t->sample_mult > 0) {
+      r.sample_mult = t->sample_mult;
+      r.sample_mult_given = true;
+    }
     if (t->segment_tiles > 0) r.segment_tiles = t->segment_tiles;
     if (t->grid > 0) r.grid = t->grid;
     r.sample_rank = t->sample_rank;
@@ -132,6 +136,15 @@ Layout make_layout(bool fused, int T, int N, int topk, int causal_offset, const 
   if (prefix > N) prefix = N;
   if (prefix < 0) prefix = 0;
   long long want = static_cast<long long>(tun.sample_mult) * topk;
+  if (tun.sample_rank == 0 && !tun.sample_mult_given && n_given == 0) {
+    // With the rank scaled to the sampling fraction the sample only has to hold a few dozen of a row's top-k
+    // keys: 64 expected ones (k' = 64 prefix / topk, rounded up to whole key tiles) already put the initial
+    // gate within a factor 1.7 of the true k/N quantile.  Short contexts then pay for far fewer sampled
+    // scores (65,536 keys, k = 2048: 2,048 instead of 6,144 per row); at 1M keys the paper's 3k stays.
+    long long enough = (64 * prefix + topk - 1) / topk;
+    enough = (enough + kTileKeys - 1) / kTileKeys * kTileKeys;
+    if (enough < want) want = enough;
+  }
   L.n_sample = static_cast<int>(want < prefix ? want : prefix);
   L.sample_stride = L.n_sample > 0 ? static_cast<int>(prefix / L.n_sample) : 1;
   if (n_given > 0) {

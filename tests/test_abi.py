@@ -106,15 +106,18 @@ def test_sample_plan_rank_keeps_misjudgement_below_1e6(lib):
                                    (1 << 22, 8192, (1 << 22) - 128), (20000, 256, 19960)]:
         n_sample, stride, rank = binding.lt_indexer_sample_plan(N, topk, causal_offset)
         prefix = min(causal_offset + 1, N)
-        assert n_sample == min(3 * topk, prefix) and stride == prefix // n_sample and 1 <= rank <= topk
+        enough = -(-(-(-64 * prefix // topk)) // 128) * 128  # 64 expected top-k keys in the sample, whole key tiles
+        assert n_sample == min(3 * topk, enough, prefix) and stride == prefix // n_sample and 1 <= rank <= topk
         if rank < topk:
             # worst case for the tail: all topk of the row's best keys lie in the sampled prefix
             tail = hypergeom.sf(rank - 1, prefix, topk, n_sample)
             assert tail < 1e-6, (N, topk, rank, tail)
+        # the paper's rule keeps the paper's sample size
         n2, s2, r2 = binding.lt_indexer_sample_plan(N, topk, causal_offset, binding.Tunables(sample_rank=-1))
-        assert (n2, s2, r2) == (n_sample, stride, topk)
+        assert (n2, s2, r2) == (min(3 * topk, prefix), prefix // min(3 * topk, prefix), topk)
+        assert binding.lt_indexer_sample_plan(N, topk, causal_offset, binding.Tunables(sample_mult=3))[0] == min(3 * topk, prefix)
         assert binding.lt_indexer_sample_plan(N, topk, causal_offset, binding.Tunables(sample_rank=7))[2] == min(7, topk)
     # a sample that is the whole prefix is exhaustive: the deterministic rank is used
-    assert binding.lt_indexer_sample_plan(4096, 2048, 4095)[2] == 2048
+    assert binding.lt_indexer_sample_plan(4096, 2048, 4095, binding.Tunables(sample_mult=3)) == (4096, 1, 2048)
     buf = (ctypes.c_int * 3)()
     assert lib.lt_indexer_sample_plan(100, 200, 50, None, buf) == -1
