@@ -392,6 +392,8 @@ def main():
     ap.add_argument("--sampler", default="strided", choices=["strided", "prev_chunk"],
                     help="prev_chunk: the sample is the 3k most frequent top-k positions of the previous chunk "
                          "(computed untimed through lt_topk_frequent; paper Sec. 3.2 'Sampling')")
+    ap.add_argument("--paged", action="store_true",
+                    help="keep the keys in a paged cache (pages of 64 keys in random order) and call lt_indexer_topk_paged")
     ap.add_argument("--aux", action="store_true",
                     help="also time the auxiliary integer ops on this step's top-k result: lt_topk_frequent and "
                          "lt_dsa_union_mask (group 64); adds an 'aux' object to the JSON line")
@@ -476,8 +478,28 @@ def main():
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")  # larger than the 126 MB L2
     stream = torch.cuda.current_stream()
 
+    page_table = None
+    if args.paged:
+        if sample_idx is not None or inp.N % 64 != 0:
+            raise SystemExit("--paged needs the default sampler and a context that is a multiple of 64 keys")
+        n_pages = inp.N // 64
+        gen = torch.Generator(device="cuda")
+        gen.manual_seed(1234)
+        page_table = torch.randperm(n_pages, device="cuda", generator=gen).to(torch.int32)
+        k_pool = torch.empty_like(k)
+        k_pool.view(n_pages, 64, inp.D)[page_table.long()] = k.view(n_pages, 64, inp.D)
+        ks_pool = None
+        if ks is not None:
+            ks_pool = torch.empty_like(ks)
+            ks_pool.view(n_pages, 64)[page_table.long()] = ks.view(n_pages, 64)
+        k, ks = k_pool, ks_pool
+        ws = torch.empty(lt.lt_indexer_topk_paged_workspace_bytes(inp.dtype, inp.T, inp.N, inp.H, inp.D, inp.topk),
+                         dtype=torch.uint8, device="cuda")
+
     def step():
-        if sample_idx is None:
+        if page_table is not None:
+            lt.lt_indexer_topk_paged(inp.dtype, q, w, k, ks, page_table, inp.N, inp.topk, inp.causal_offset, out_idx, out_score, ws)
+        elif sample_idx is None:
             lt.lt_indexer_topk_ex(inp.dtype, q, w, k, ks, inp.topk, inp.causal_offset, out_idx, out_score, ws)
         else:
             lt.lt_indexer_topk_sampled(inp.dtype, q, w, k, ks, inp.topk, inp.causal_offset, sample_idx, out_idx, out_score, ws)
@@ -574,7 +596,8 @@ def main():
         "dtype": "fp8_e4m3" if fp8 else inp.dtype, "data": "synthetic",
         "config": {"workload": args.workload, "T": inp.T, "N": inp.N, "H": inp.H, "D": inp.D, "topk": inp.topk,
                    "causal_offset": inp.causal_offset, "valid_pairs": pairs, "parallelism": f"replicas x{world}",
-                   "l2": "flushed between timed iterations (256 MiB write)", "workspace_bytes": int(ws.numel())},
+                   "l2": "flushed between timed iterations (256 MiB write)", "workspace_bytes": int(ws.numel()),
+                   "key_layout": "paged (64-key pages, random order)" if page_table is not None else "dense"},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms / e2e_steps},
@@ -590,7 +613,7 @@ def main():
     if args.aux:
         line["aux"] = time_aux_ops(torch, lt, out_idx, inp, peaks["hbm_gbs"], peak_kind)
 
-    if not args.no_unfused:
+    if not args.no_unfused and page_table is None:
         # in-repo unfused GPU baseline: dense scores to HBM in row sub-chunks, then a full-row radix select
         buf = torch.empty(256 + (args.unfused_budget_mb << 20), dtype=torch.uint8, device="cuda")
 

@@ -152,6 +152,27 @@ size_t lt_indexer_topk_sampled_workspace_bytes(int dtype, int T, int N, int H, i
                                                const lt_tunables* tunables);
 
 /*
+ * Fused indexer top-k over a PAGED key cache (serving layout; the paper's kernel reads the cache of its
+ * serving engine, Sec. 4.1).  Keys live in a pool of pages of LT_PAGE_KEYS = 64 consecutive rows:
+ *   k_pool        device, [pool_rows][D] (bf16 or e4m3), pool_rows a multiple of 64
+ *   k_scale_pool  device, [pool_rows] fp32 (e4m3 only), indexed like k_pool
+ *   page_table    device, n_pages int32: keys 64 j .. 64 j + 63 of the context are pool rows
+ *                 64 page_table[j] .. 64 page_table[j] + 63; n_pages * 64 >= N; entries must be valid
+ *                 page numbers (0 <= page_table[j] < pool_rows / 64)
+ * Everything else as lt_indexer_topk_ex, and the outputs are bit-identical to lt_indexer_topk_ex on the
+ * same keys laid out densely.  Only shapes of the tensor-core path (H = 64, D = 128, bf16 or e4m3);
+ * LT_ERR_UNSUPPORTED otherwise.  workspace: lt_indexer_topk_paged_workspace_bytes(...) bytes (the sampled
+ * keys are gathered into it: a strided view cannot reach a paged cache).
+ */
+#define LT_PAGE_KEYS 64
+int lt_indexer_topk_paged(int dtype, const void* q, const float* w, const void* k_pool, const float* k_scale_pool,
+                          const int32_t* page_table, int n_pages, long long pool_rows,
+                          int T, int N, int H, int D, int topk, int causal_offset,
+                          int32_t* out_idx, float* out_score,
+                          void* workspace, size_t workspace_bytes, const lt_tunables* tunables, void* stream);
+size_t lt_indexer_topk_paged_workspace_bytes(int dtype, int T, int N, int H, int D, int topk, const lt_tunables* tunables);
+
+/*
  * The n_out positions that occur most often in a chunk's top-k index matrix (paper Sec. 3.2
  * "Sampling": the previous-chunk sampler), ordered by (count descending, position ascending);
  * positions that never occur (count 0) fill the tail in ascending order.

@@ -66,6 +66,11 @@ def load() -> ctypes.CDLL:
     lib.lt_indexer_topk_sampled.restype = i
     lib.lt_indexer_topk_sampled_workspace_bytes.argtypes = [i, i, i, i, i, i, i, ctypes.POINTER(Tunables)]
     lib.lt_indexer_topk_sampled_workspace_bytes.restype = sz
+    lib.lt_indexer_topk_paged.argtypes = [i, vp, fp, vp, fp, ip, i, ctypes.c_longlong, i, i, i, i, i, i, ip, fp, vp, sz,
+                                          ctypes.POINTER(Tunables), vp]
+    lib.lt_indexer_topk_paged.restype = i
+    lib.lt_indexer_topk_paged_workspace_bytes.argtypes = [i, i, i, i, i, i, ctypes.POINTER(Tunables)]
+    lib.lt_indexer_topk_paged_workspace_bytes.restype = sz
     lib.lt_topk_frequent.argtypes = [ip, i, i, i, i, ip, ip, vp, sz, vp]
     lib.lt_topk_frequent.restype = i
     lib.lt_topk_frequent_workspace_bytes.argtypes = [i]
@@ -182,6 +187,25 @@ def lt_indexer_topk_sampled(dtype, q, w, k, k_scale, topk: int, causal_offset: i
                                           _ptr(workspace), workspace.numel() * workspace.element_size(),
                                           ctypes.byref(tunables) if tunables else None, _stream(stream)),
            "lt_indexer_topk_sampled")
+
+
+def lt_indexer_topk_paged_workspace_bytes(dtype, T: int, N: int, H: int, D: int, topk: int,
+                                          tunables: Optional[Tunables] = None) -> int:
+    return int(load().lt_indexer_topk_paged_workspace_bytes(dtype_code(dtype), T, N, H, D, topk,
+                                                            ctypes.byref(tunables) if tunables else None))
+
+
+def lt_indexer_topk_paged(dtype, q, w, k_pool, k_scale_pool, page_table, N: int, topk: int, causal_offset: int, out_idx,
+                          out_score, workspace, tunables: Optional[Tunables] = None, stream=None) -> None:
+    """lt_indexer_topk_ex over a paged key cache: k_pool [pool_rows, D], page_table int32 [n_pages] (pages of 64 keys)."""
+    T, H, D = q.shape
+    pool_rows, D2 = k_pool.shape
+    if D2 != D:
+        raise ValueError("q and k_pool disagree on D")
+    _check(load().lt_indexer_topk_paged(dtype_code(dtype), _ptr(q), _ptr(w), _ptr(k_pool), _ptr(k_scale_pool), _ptr(page_table),
+                                        page_table.numel(), pool_rows, T, N, H, D, topk, causal_offset, _ptr(out_idx),
+                                        _ptr(out_score), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                        ctypes.byref(tunables) if tunables else None, _stream(stream)), "lt_indexer_topk_paged")
 
 
 def lt_topk_frequent_workspace_bytes(N: int) -> int:

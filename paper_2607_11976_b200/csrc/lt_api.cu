@@ -97,8 +97,9 @@ struct Layout {
 
 // n_given > 0: the caller provides that many sample positions (lt_indexer_topk_sampled); their keys are
 // gathered into a dense buffer of the workspace (key_row_bytes each) and scored from there.
+// gather_default: the default strided sample is gathered too (paged key cache: a strided view cannot reach it).
 Layout make_layout(bool fused, int T, int N, int topk, int causal_offset, const Tun& tun, int n_given = 0,
-                   int key_row_bytes = 0) {
+                   int key_row_bytes = 0, bool gather_default = false) {
   Layout L{};
   L.fused = fused;
   size_t off = 0;
@@ -166,10 +167,11 @@ Layout make_layout(bool fused, int T, int N, int topk, int causal_offset, const 
   }
   L.sample = off;
   off = align_up(off + static_cast<size_t>(T) * (L.n_sample > 0 ? L.n_sample : 1) * 4);
+  const int gather_rows = n_given > 0 ? n_given : (gather_default ? L.n_sample : 0);
   L.gather_k = off;
-  off = align_up(off + static_cast<size_t>(n_given) * key_row_bytes);
+  off = align_up(off + static_cast<size_t>(gather_rows) * key_row_bytes);
   L.gather_scale = off;
-  off = align_up(off + static_cast<size_t>(n_given) * 4);
+  off = align_up(off + static_cast<size_t>(gather_rows) * 4);
   long long cap = static_cast<long long>(tun.cap_mult) * topk;
   L.cap = static_cast<int>(cap > N ? N : cap);
   L.cand = off;
@@ -256,7 +258,8 @@ size_t elem_bytes(int dtype) { return dtype == LT_DTYPE_F32 ? 4 : (dtype == LT_D
 
 int topk_impl(int dtype, const void* q, const float* w, const void* k, const float* k_scale, int T, int N, int H, int D, int topk,
               int causal_offset, int32_t* out_idx, float* out_score, void* workspace, size_t workspace_bytes,
-              const lt_tunables* tunables, cudaStream_t stream, const int32_t* sample_idx = nullptr, int n_given = 0) {
+              const lt_tunables* tunables, cudaStream_t stream, const int32_t* sample_idx = nullptr, int n_given = 0,
+              const int* page_table = nullptr, int n_pages = 0, long long pool_rows = 0) {
   int rc = check_problem(dtype, q, w, k, k_scale, T, N, H, D);
   if (rc != LT_OK) return rc;
   if (out_idx == nullptr || topk <= 0 || topk > N || topk > LT_MAX_TOPK) return LT_ERR_INVALID_ARG;
@@ -264,7 +267,10 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
   const bool fused = use_fused(tun, dtype, H, D);
   if (tun.path == LT_PATH_FUSED && !fused) return LT_ERR_UNSUPPORTED;
   const int key_row_bytes = static_cast<int>(static_cast<size_t>(D) * elem_bytes(dtype));
-  const Layout L = make_layout(fused, T, N, topk, causal_offset, tun, n_given, key_row_bytes);
+  const bool paged = page_table != nullptr;
+  if (paged && !fused) return LT_ERR_UNSUPPORTED;
+  const Layout L = make_layout(fused, T, N, topk, causal_offset, tun, n_given, key_row_bytes, paged);
+  const long long key_rows = paged ? pool_rows : N;  // rows the key tensor map covers
   if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) != 0 || workspace_bytes < L.total)
     return LT_ERR_WORKSPACE;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
@@ -294,17 +300,21 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
   mark_phase(0, stream);
   const void* sample_keys = k;
   const float* sample_scale = k_scale;
-  if (n_given > 0) {
-    LT_LAUNCH(launch_gather_keys(k, k_scale, sample_idx, n_given, N, key_row_bytes, ws + L.gather_k,
-                                 reinterpret_cast<float*>(ws + L.gather_scale), stream));
+  long long sample_pitch = static_cast<long long>(L.sample_stride) * D;
+  long long sample_ks_stride = L.sample_stride;
+  if ((n_given > 0 || paged) && L.n_sample > 0) {
+    LT_LAUNCH(launch_gather_keys(k, k_scale, n_given > 0 ? sample_idx : nullptr, L.sample_stride, L.n_sample, N, key_row_bytes,
+                                 page_table, ws + L.gather_k, reinterpret_cast<float*>(ws + L.gather_scale), stream));
     sample_keys = ws + L.gather_k;
     if (k_scale != nullptr) sample_scale = reinterpret_cast<const float*>(ws + L.gather_scale);
+    sample_pitch = D;
+    sample_ks_stride = 1;
   }
   if (L.n_sample > 0) {
     ScanParams p{};
     p.w = w;
     p.k_scale = sample_scale;
-    p.ks_stride = L.sample_stride;
+    p.ks_stride = sample_ks_stride;
     p.T = T;
     p.row_begin = 0;
     p.row_end = T;
@@ -316,8 +326,7 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
     p.dump = sample;
     p.dump_ld = L.n_sample;
     p.ctl = ctl;
-    LT_LAUNCH(launch_scan_mma(dtype, kModeDump, q, T, sample_keys, L.n_sample, static_cast<long long>(L.sample_stride) * D, p, grid,
-                              stream));
+    LT_LAUNCH(launch_scan_mma(dtype, kModeDump, q, T, sample_keys, L.n_sample, sample_pitch, p, grid, stream));
   }
   mark_phase(1, stream);
   LT_LAUNCH(launch_sample_stats(sample, T, L.n_sample, L.sample_rank, smin, width, thr, stream));
@@ -344,8 +353,10 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
     p.hist = hist;
     p.cand = cand;
     p.cap = L.cap;
+    p.page_table = page_table;
+    p.n_pages = n_pages;
     p.ctl = ctl;
-    LT_LAUNCH(launch_scan_mma(dtype, kModeFilter, q, T, k, N, D, p, grid, stream));
+    LT_LAUNCH(launch_scan_mma(dtype, kModeFilter, q, T, k, key_rows, D, p, grid, stream));
   }
 
   // 3. final select over the survivors; rows it cannot finish exactly are flagged
@@ -394,8 +405,10 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
     p.fb_blocks = &ctl->fb_blocks;
     p.fb_round_base = r * L.fb_slots;
     p.fb_slots = L.fb_slots;
+    p.page_table = page_table;
+    p.n_pages = n_pages;
     p.ctl = ctl;
-    LT_LAUNCH(launch_scan_mma(dtype, kModeDump, q, T, k, N, D, p, grid, stream));
+    LT_LAUNCH(launch_scan_mma(dtype, kModeDump, q, T, k, key_rows, D, p, grid, stream));
     SelectRowsParams sp{};
     sp.scores = scratch;
     sp.ld = N;
@@ -497,6 +510,26 @@ size_t lt_indexer_topk_sampled_workspace_bytes(int dtype, int T, int N, int H, i
   const Tun tun = resolve_tunables(tunables);
   return make_layout(use_fused(tun, dtype, H, D), T, N, topk, N - 1, tun, n_sample,
                      static_cast<int>(static_cast<size_t>(D) * elem_bytes(dtype))).total;
+}
+
+int lt_indexer_topk_paged(int dtype, const void* q, const float* w, const void* k_pool, const float* k_scale_pool,
+                          const int32_t* page_table, int n_pages, long long pool_rows, int T, int N, int H, int D, int topk,
+                          int causal_offset, int32_t* out_idx, float* out_score, void* workspace, size_t workspace_bytes,
+                          const lt_tunables* tunables, void* stream) {
+  if (page_table == nullptr || n_pages <= 0 || pool_rows <= 0 || pool_rows % kPageKeys != 0 ||
+      static_cast<long long>(n_pages) * kPageKeys < N)
+    return LT_ERR_INVALID_ARG;
+  return topk_impl(dtype, q, w, k_pool, k_scale_pool, T, N, H, D, topk, causal_offset, out_idx, out_score, workspace,
+                   workspace_bytes, tunables, static_cast<cudaStream_t>(stream), nullptr, 0, page_table, n_pages, pool_rows);
+}
+
+size_t lt_indexer_topk_paged_workspace_bytes(int dtype, int T, int N, int H, int D, int topk, const lt_tunables* tunables) {
+  if ((dtype != LT_DTYPE_BF16 && dtype != LT_DTYPE_E4M3) || T <= 0 || N <= 0 || H <= 0 || D <= 0 || topk <= 0 || topk > N ||
+      topk > LT_MAX_TOPK)
+    return 0;
+  const Tun tun = resolve_tunables(tunables);
+  if (!use_fused(tun, dtype, H, D)) return 0;
+  return make_layout(true, T, N, topk, N - 1, tun, 0, static_cast<int>(static_cast<size_t>(D) * elem_bytes(dtype)), true).total;
 }
 
 size_t lt_topk_frequent_workspace_bytes(int N) {

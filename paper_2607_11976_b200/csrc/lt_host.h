@@ -42,8 +42,13 @@ struct ScanParams {
   const int* fb_blocks;    // device counter: entries in fb_list
   int fb_round_base;
   int fb_slots;
+  // paged key cache (null: keys are one dense matrix): logical page j of 64 keys is physical page page_table[j] of
+  // the pool the key tensor map covers; k_scale is then indexed by physical row
+  const int* page_table;
+  int n_pages;
   Control* ctl;
 };
+constexpr int kPageKeys = 64;  // keys per page of a paged key cache
 
 bool scan_mma_supported(int dtype, int H, int D);
 
@@ -133,9 +138,10 @@ cudaError_t launch_count_positions(const int32_t* idx, long long n, int N, unsig
 // in place: counts[i] (u32) -> the same value as fp32 bits
 cudaError_t launch_counts_to_float(unsigned int* counts, int N, cudaStream_t stream);
 cudaError_t launch_float_to_counts(const float* f, int n, int32_t* out, cudaStream_t stream);
-// dense copy of the key rows (row_bytes each, multiple of 16) and scales at the sampled positions
-cudaError_t launch_gather_keys(const void* k, const float* k_scale, const int32_t* sample_idx, int n_sample, int N,
-                               int row_bytes, void* out_k, float* out_scale, cudaStream_t stream);
+// dense copy of the key rows (row_bytes each, multiple of 16) and scales at the sampled positions (sample_idx, or
+// j * stride when it is null); page_table (or null) translates positions to physical rows of a paged key cache
+cudaError_t launch_gather_keys(const void* k, const float* k_scale, const int32_t* sample_idx, long long stride, int n_sample,
+                               int N, int row_bytes, const int* page_table, void* out_k, float* out_scale, cudaStream_t stream);
 
 // ---- lt_dsa_union.cu ------------------------------------------------------------------------
 // LiteDSA union list + membership masks of consecutive groups of `group` rows (paper Sec. 3.3).

@@ -44,19 +44,22 @@ __global__ void __launch_bounds__(256) float_to_counts_kernel(const float* __res
   if (i < n) out[i] = static_cast<int32_t>(f[i]);
 }
 
-// out_k[j] = key row sample_idx[j] (row_bytes bytes, a multiple of 16), out_scale[j] = its scale.
-// One 16-byte piece per thread; positions outside [0, N) are read as position 0.
+// out_k[j] = key row at position sample_idx[j] (or j * stride when no list is given), row_bytes bytes (a
+// multiple of 16); out_scale[j] = its scale.  One 16-byte piece per thread; positions outside [0, N) are read as
+// position 0.  With a paged key cache the position is translated to its physical row first.
 __global__ void __launch_bounds__(256) gather_keys_kernel(const uint8_t* __restrict__ k, const float* __restrict__ k_scale,
-                                                          const int32_t* __restrict__ sample_idx, int n_sample, int N,
-                                                          int row_bytes, uint8_t* __restrict__ out_k,
+                                                          const int32_t* __restrict__ sample_idx, long long stride,
+                                                          int n_sample, int N, int row_bytes,
+                                                          const int* __restrict__ page_table, uint8_t* __restrict__ out_k,
                                                           float* __restrict__ out_scale) {
   const int pieces = row_bytes >> 4;
   const long long g = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   const long long j = g / pieces;
   const int piece = static_cast<int>(g - j * pieces);
   if (j >= n_sample) return;
-  int s = __ldg(sample_idx + j);
-  if (static_cast<unsigned int>(s) >= static_cast<unsigned int>(N)) s = 0;
+  long long s = sample_idx != nullptr ? static_cast<long long>(__ldg(sample_idx + j)) : j * stride;
+  if (s < 0 || s >= N) s = 0;
+  if (page_table != nullptr) s = static_cast<long long>(__ldg(page_table + s / kPageKeys)) * kPageKeys + s % kPageKeys;
   const uint4 v = __ldg(reinterpret_cast<const uint4*>(k + static_cast<size_t>(s) * row_bytes) + piece);
   reinterpret_cast<uint4*>(out_k + static_cast<size_t>(j) * row_bytes)[piece] = v;
   if (piece == 0 && k_scale != nullptr) out_scale[j] = __ldg(k_scale + s);
@@ -83,11 +86,12 @@ cudaError_t launch_float_to_counts(const float* f, int n, int32_t* out, cudaStre
   return cudaGetLastError();
 }
 
-cudaError_t launch_gather_keys(const void* k, const float* k_scale, const int32_t* sample_idx, int n_sample, int N,
-                               int row_bytes, void* out_k, float* out_scale, cudaStream_t stream) {
+cudaError_t launch_gather_keys(const void* k, const float* k_scale, const int32_t* sample_idx, long long stride, int n_sample,
+                               int N, int row_bytes, const int* page_table, void* out_k, float* out_scale, cudaStream_t stream) {
   const long long threads = static_cast<long long>(n_sample) * (row_bytes >> 4);
   gather_keys_kernel<<<static_cast<int>((threads + 255) / 256), 256, 0, stream>>>(
-      static_cast<const uint8_t*>(k), k_scale, sample_idx, n_sample, N, row_bytes, static_cast<uint8_t*>(out_k), out_scale);
+      static_cast<const uint8_t*>(k), k_scale, sample_idx, stride, n_sample, N, row_bytes, page_table,
+      static_cast<uint8_t*>(out_k), out_scale);
   return cudaGetLastError();
 }
 

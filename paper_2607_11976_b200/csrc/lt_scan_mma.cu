@@ -123,6 +123,13 @@ __device__ __forceinline__ bool resolve_item(const ScanParams& p, int n_blocks, 
   return it.tile_lo < it.tile_hi;
 }
 
+// Where the scale of view key s lives: at s * ks_stride, or with a paged key cache at the key's physical row.
+template <bool kPaged>
+__device__ __forceinline__ size_t scale_index(const ScanParams& p, int s) {
+  if (kPaged) return static_cast<size_t>(__ldg(p.page_table + (s / kPageKeys))) * kPageKeys + static_cast<size_t>(s % kPageKeys);
+  return static_cast<size_t>(s) * p.ks_stride;
+}
+
 // ---- Eq. 1 for one key against one query ------------------------------------------------------
 // 32 TMEM columns (per-head dots) -> ReLU -> weighted sum, accumulated into four packed fp32 pairs
 // (eight independent chains).  Head h lands in pair (h / 2) % 4, lane h % 2; combine() fixes the
@@ -218,7 +225,7 @@ __device__ __forceinline__ void flush_stage(const uint2* list, int count, const 
   __syncwarp();
 }
 
-template <bool kFp8, int kMode>
+template <bool kFp8, int kMode, bool kPaged>
 __global__ void __launch_bounds__(kThreads, 1)
 scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k, const ScanParams p) {
   using C = Cfg<kFp8>;
@@ -299,9 +306,21 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           ok = mbar_wait<40>(smem_u32(&st->bar_empty[stage]), phase ^ 1, abort_flag);
           if (!ok) break;
           mbar_arrive_expect_tx(smem_u32(&st->bar_full[stage]), C::kStageBytes);
-          for (int hf = 0; hf < C::kHalves; ++hf)
-            tma_load_2d(k_base + stage * C::kStageBytes + hf * kSwizzleTile, &tm_k, hf * C::kElemsPerRow128,
-                        tile * kTileKeys, smem_u32(&st->bar_full[stage]));
+          if (!kPaged) {
+            for (int hf = 0; hf < C::kHalves; ++hf)
+              tma_load_2d(k_base + stage * C::kStageBytes + hf * kSwizzleTile, &tm_k, hf * C::kElemsPerRow128,
+                          tile * kTileKeys, smem_u32(&st->bar_full[stage]));
+          } else {
+            // paged key cache: a tile is two pages of 64 keys, each wherever the page table says (the map's
+            // box is then 64 rows); pages past the end of the table are read from page 0 and masked later
+            for (int pg = 0; pg < kTileKeys / kPageKeys; ++pg) {
+              const int lp = tile * (kTileKeys / kPageKeys) + pg;
+              const int phys = lp < p.n_pages ? __ldg(p.page_table + lp) : 0;
+              for (int hf = 0; hf < C::kHalves; ++hf)
+                tma_load_2d(k_base + stage * C::kStageBytes + hf * kSwizzleTile + pg * kPageKeys * 128, &tm_k,
+                            hf * C::kElemsPerRow128, phys * kPageKeys, smem_u32(&st->bar_full[stage]));
+            }
+          }
           if (++stage == C::kStages) {
             stage = 0;
             phase ^= 1;
@@ -470,7 +489,7 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         float ks_next = 1.f;
         {
           const int s0 = it.tile_lo * kTileKeys + key_in_tile;
-          if (has_scale && s0 < p.n_keys) ks_next = __ldg(p.k_scale + static_cast<size_t>(s0) * p.ks_stride);
+          if (has_scale && s0 < p.n_keys) ks_next = __ldg(p.k_scale + scale_index<kPaged>(p, s0));
         }
         for (int tile = it.tile_lo; tile < it.tile_hi && ok; ++tile) {
           const int s = tile * kTileKeys + key_in_tile;
@@ -478,7 +497,7 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           {
             const int s1 = s + kTileKeys;
             if (has_scale && tile + 1 < it.tile_hi && s1 < p.n_keys)
-              ks_next = __ldg(p.k_scale + static_cast<size_t>(s1) * p.ks_stride);
+              ks_next = __ldg(p.k_scale + scale_index<kPaged>(p, s1));
           }
           // keys of this tile that some row of the block may not see (diagonal or ragged last tile)
           const bool partial = (tile + 1) * kTileKeys > vis_first;
@@ -600,13 +619,19 @@ bool make_map(CUtensorMap* map, bool fp8, const void* base, uint64_t rows, uint6
   return r == CUDA_SUCCESS;
 }
 
+template <bool kFp8, int kMode, bool kPaged>
+cudaError_t launch_one(const CUtensorMap& tq, const CUtensorMap& tk, const ScanParams& p, int grid, cudaStream_t stream) {
+  constexpr int bytes = smem_bytes<kFp8>();
+  cudaError_t e = cudaFuncSetAttribute(scan_kernel<kFp8, kMode, kPaged>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return e;
+  scan_kernel<kFp8, kMode, kPaged><<<grid, kThreads, bytes, stream>>>(tq, tk, p);
+  return cudaGetLastError();
+}
+// the paged variant is a separate instantiation so that the dense kernels carry none of its address arithmetic
 template <bool kFp8, int kMode>
 cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const ScanParams& p, int grid, cudaStream_t stream) {
-  constexpr int bytes = smem_bytes<kFp8>();
-  cudaError_t e = cudaFuncSetAttribute(scan_kernel<kFp8, kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  if (e != cudaSuccess) return e;
-  scan_kernel<kFp8, kMode><<<grid, kThreads, bytes, stream>>>(tq, tk, p);
-  return cudaGetLastError();
+  return p.page_table != nullptr ? launch_one<kFp8, kMode, true>(tq, tk, p, grid, stream)
+                                 : launch_one<kFp8, kMode, false>(tq, tk, p, grid, stream);
 }
 
 }  // namespace
@@ -621,7 +646,9 @@ cudaError_t launch_scan_mma(int dtype, int mode, const void* q, int T, const voi
   const size_t esz = fp8 ? 1 : 2;
   CUtensorMap tq, tk;
   if (!make_map(&tq, fp8, q, static_cast<uint64_t>(T) * kH, kD * esz, 256)) return cudaErrorInvalidValue;
-  if (!make_map(&tk, fp8, k, static_cast<uint64_t>(n_keys_view), static_cast<uint64_t>(key_pitch_elems) * esz, 128))
+  // dense keys: one 128-row box per tile; paged keys (k = the page pool, n_keys_view = its rows): 64-row boxes
+  if (!make_map(&tk, fp8, k, static_cast<uint64_t>(n_keys_view), static_cast<uint64_t>(key_pitch_elems) * esz,
+                p.page_table != nullptr ? kPageKeys : 128))
     return cudaErrorInvalidValue;
   if (fp8) {
     return mode == kModeFilter ? launch<true, kModeFilter>(tq, tk, p, grid, stream) : launch<true, kModeDump>(tq, tk, p, grid, stream);
