@@ -164,9 +164,48 @@ def time_oracle(inp, budget_s: float, max_rows: int = 64):
     return pairs / dt, done_rows, pairs, dt
 
 
+def run_reference_knn(args):
+    """`--impl reference` for the k-NN workloads: the fp64 oracle on a few query rows per step."""
+    from oracle import knn_topk
+    from workloads import make_knn
+
+    inp = make_knn(args.workload, N=args.knn_corpus or None)
+    np.matmul(np.ones((64, 64)), np.ones((64, 64)))
+    rows_per_step = 2
+    for _ in range(min(args.warmup, 1)):
+        knn_topk(inp.q, inp.x, inp.topk, rows=[0])
+    vals = []
+    budget = args.cpu_budget / max(1, args.steps)
+    for s_i in range(args.steps):
+        t0 = time.perf_counter()
+        done = 0
+        while done < inp.T and (done == 0 or time.perf_counter() - t0 < budget):
+            r0 = (s_i * 16 + done) % inp.T
+            knn_topk(inp.q, inp.x, inp.topk, rows=list(range(r0, min(inp.T, r0 + rows_per_step))))
+            done += rows_per_step
+        dt = time.perf_counter() - t0
+        vals.append((done * inp.N / dt, dt, done))
+    value = statistics.mean(v for v, _, _ in vals)
+    sample = f"{vals[-1][2]} query rows x the whole corpus per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": statistics.mean(dt for _, dt, _ in vals) * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "T": inp.T, "N": inp.N, "D": inp.D, "topk": inp.topk,
+                   "note": "CPU oracle (numpy fp64 matmul + full sort) on a bounded row sample of the workload"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
 def run_reference(args, rank: int):
     """`--impl reference`: the CPU oracle on the host cores, rank 0 only."""
     if rank != 0:
+        return
+    if args.workload.startswith("knn"):
+        run_reference_knn(args)
         return
     from workloads import make_config
 
