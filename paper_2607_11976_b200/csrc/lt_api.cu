@@ -534,7 +534,7 @@ size_t lt_indexer_topk_paged_workspace_bytes(int dtype, int T, int N, int H, int
 
 size_t lt_topk_frequent_workspace_bytes(int N) {
   if (N <= 0) return 0;
-  return align_up(static_cast<size_t>(N) * 4) + align_up(static_cast<size_t>(LT_MAX_TOPK) * 4);
+  return align_up(static_cast<size_t>(N) * 4) + align_up(rank_scratch_bytes(LT_MAX_TOPK));
 }
 
 int lt_topk_frequent(const int32_t* idx, int T, int topk, int N, int n_out, int32_t* out_pos, int32_t* out_count,
@@ -548,26 +548,11 @@ int lt_topk_frequent(const int32_t* idx, int T, int topk, int N, int n_out, int3
     return LT_ERR_WORKSPACE;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   unsigned int* counts = reinterpret_cast<unsigned int*>(ws);
-  float* sel_score = reinterpret_cast<float*>(ws + align_up(static_cast<size_t>(N) * 4));
+  void* scratch = ws + align_up(static_cast<size_t>(N) * 4);
   LT_CUDA(cudaMemsetAsync(counts, 0, static_cast<size_t>(N) * 4, stream));
   LT_LAUNCH(launch_count_positions(idx, static_cast<long long>(T) * topk, N, counts, stream));
-  // a position occurs at most once per row, and in any case at most T * topk < 2^24 * 2^13 times; counts up
-  // to 2^24 are exact in fp32, larger ones (only possible with repeated positions inside a row) would still
-  // rank monotonically but lose their low bits, so such matrices are outside the contract
-  LT_LAUNCH(launch_counts_to_float(counts, N, stream));
-  SelectRowsParams sp{};
-  sp.scores = reinterpret_cast<const float*>(counts);
-  sp.ld = N;
-  sp.n_blocks = 1;
-  sp.row_begin = 0;
-  sp.T = 1;
-  sp.N = N;
-  sp.topk = n_out;
-  sp.causal_offset = N - 1;
-  sp.out_idx = out_pos;
-  sp.out_score = sel_score;
-  LT_LAUNCH(launch_select_rows(sp, stream));
-  if (out_count != nullptr) LT_LAUNCH(launch_float_to_counts(sel_score, n_out, out_count, stream));
+  // rank the N (count, position) pairs with a grid-wide radix select and sort the n_out winners
+  LT_LAUNCH(launch_rank_counts(counts, N, n_out, scratch, out_pos, out_count, stream));
   return LT_OK;
 }
 

@@ -1,5 +1,5 @@
 // Previous-chunk sampler (paper Sec. 3.2 "Sampling"): count how often each key position occurs in a
-// chunk's top-k result, and gather the keys of a caller-provided sample into a dense buffer that the
+// chunk's top-k result, rank the counts, and gather the keys of a caller-provided sample into a dense buffer that the
 // scan kernel can score through an ordinary tensor map.  Integer / byte work only.
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -31,17 +31,123 @@ __global__ void __launch_bounds__(256) count_positions_kernel(const int32_t* __r
   }
 }
 
-// counts (u32) -> the same numbers as fp32, in place, so that the full-row select can rank them.
-// Exact: a count is at most T * topk entries of one matrix, and the launcher rejects matrices with
-// more than 2^24 entries per position bound (T <= 2^24).
-__global__ void __launch_bounds__(256) counts_to_float_kernel(unsigned int* __restrict__ counts, int N) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < N) counts[i] = __float_as_uint(static_cast<float>(counts[i]));
+// ---- ranking the counts: top n_out of the N distinct 64-bit keys (count << 32 | ~position) ---------------------
+// A grid-wide MSB radix select, one launch per 8-bit digit: every CTA histograms the digit of the keys that
+// still match the prefix found so far (per-thread run-length aggregation: neighbouring positions mostly share
+// the digit), adds its 256 counters to the global histogram, and the last CTA to finish picks the digit in
+// which the count from the top reaches the number of keys still wanted.  The keys are distinct (the position
+// is part of them), so after eight digits the prefix IS the n_out-th largest key and no tie needs ranking.
+struct RankState {
+  unsigned int hist[256];
+  unsigned long long prefix;
+  unsigned int remaining;
+  unsigned int done;
+  unsigned int n_written;
+  unsigned int pad[3];
+};
+
+__device__ __forceinline__ unsigned long long rank_key(unsigned int count, unsigned int pos) {
+  return (static_cast<unsigned long long>(count) << 32) | (0xffffffffu - pos);
 }
 
-__global__ void __launch_bounds__(256) float_to_counts_kernel(const float* __restrict__ f, int n, int32_t* __restrict__ out) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) out[i] = static_cast<int32_t>(f[i]);
+__global__ void __launch_bounds__(256) rank_pass_kernel(const unsigned int* __restrict__ counts, int N, RankState* st, int pass,
+                                                         int want) {
+  __shared__ unsigned int hist[256];
+  __shared__ bool last;
+  const int shift = 56 - 8 * pass;
+  const unsigned long long mask = pass == 0 ? 0ull : (~0ull << (shift + 8));
+  const unsigned long long prefix = st->prefix;
+  hist[threadIdx.x] = 0;
+  __syncthreads();
+  unsigned int run_digit = 0x100u, run_len = 0;
+  // each CTA walks one contiguous range of positions with coalesced loads; a thread's consecutive keys are
+  // 256 positions apart, which still share their leading digits (the count's high bytes)
+  const int per_thread = (N + gridDim.x * blockDim.x - 1) / (gridDim.x * blockDim.x);
+  const long long first = static_cast<long long>(blockIdx.x) * blockDim.x * per_thread + threadIdx.x;
+  for (int j = 0; j < per_thread; ++j) {
+    const long long i = first + static_cast<long long>(j) * blockDim.x;
+    if (i >= N) break;
+    const unsigned long long key = rank_key(__ldg(counts + i), static_cast<unsigned int>(i));
+    if ((key & mask) != prefix) continue;
+    const unsigned int digit = static_cast<unsigned int>(key >> shift) & 255u;
+    if (digit == run_digit) {
+      ++run_len;
+    } else {
+      if (run_len > 0) atomicAdd(&hist[run_digit], run_len);
+      run_digit = digit;
+      run_len = 1;
+    }
+  }
+  if (run_len > 0) atomicAdd(&hist[run_digit], run_len);
+  __syncthreads();
+  if (hist[threadIdx.x] != 0) atomicAdd(&st->hist[threadIdx.x], hist[threadIdx.x]);
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) last = atomicAdd(&st->done, 1u) == gridDim.x - 1;
+  __syncthreads();
+  if (!last) return;
+  __threadfence();
+  // the complete histogram comes back with one load per thread (a single thread walking it in global memory
+  // would pay 256 dependent L2 round trips)
+  hist[threadIdx.x] = __ldcg(&st->hist[threadIdx.x]);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned int remaining = pass == 0 ? static_cast<unsigned int>(want) : st->remaining;
+    unsigned int cum = 0;
+    int digit = 0;
+    for (int d = 255; d >= 0; --d) {
+      const unsigned int c = hist[d];
+      if (cum + c >= remaining) {
+        digit = d;
+        break;
+      }
+      cum += c;
+    }
+    st->remaining = remaining - cum;
+    st->prefix = prefix | (static_cast<unsigned long long>(digit) << shift);
+    st->done = 0;
+  }
+  __syncthreads();
+  st->hist[threadIdx.x] = 0;
+}
+
+// every key at or above the n_out-th largest goes to the list (any order; exactly n_out of them)
+__global__ void __launch_bounds__(256) rank_collect_kernel(const unsigned int* __restrict__ counts, int N, RankState* st,
+                                                            unsigned long long* __restrict__ keys, int n_out) {
+  const unsigned long long kth = st->prefix;
+  const int lane = threadIdx.x & 31;
+  const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+  const long long n_round = (N + stride - 1) / stride * stride;
+  for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < n_round; i += stride) {
+    unsigned long long key = 0;
+    bool take = false;
+    if (i < N) {
+      key = rank_key(__ldg(counts + i), static_cast<unsigned int>(i));
+      take = key >= kth;
+    }
+    const unsigned int ballot = __ballot_sync(0xffffffffu, take);
+    if (ballot != 0) {
+      unsigned int base = 0;
+      if (lane == 0) base = atomicAdd(&st->n_written, static_cast<unsigned int>(__popc(ballot)));
+      base = __shfl_sync(0xffffffffu, base, 0);
+      const unsigned int pos = base + __popc(ballot & ((1u << lane) - 1u));
+      if (take && pos < static_cast<unsigned int>(n_out)) keys[pos] = key;
+    }
+  }
+}
+
+// one CTA: sort the n_out keys (descending = count descending, position ascending) and write the outputs
+__global__ void __launch_bounds__(1024) rank_sort_kernel(const unsigned long long* __restrict__ keys, int n_out,
+                                                          int32_t* __restrict__ out_pos, int32_t* __restrict__ out_count) {
+  extern __shared__ uint64_t sel[];
+  const int n = next_pow2(n_out < 2 ? 2 : n_out);
+  for (int i = threadIdx.x; i < n; i += blockDim.x) sel[i] = i < n_out ? keys[i] : 0ull;
+  __syncthreads();
+  bitonic_sort_desc(sel, n, threadIdx.x, blockDim.x);
+  for (int i = threadIdx.x; i < n_out; i += blockDim.x) {
+    out_pos[i] = static_cast<int32_t>(0xffffffffu - static_cast<unsigned int>(sel[i]));
+    if (out_count != nullptr) out_count[i] = static_cast<int32_t>(sel[i] >> 32);
+  }
 }
 
 // out_k[j] = key row at position sample_idx[j] (or j * stride when no list is given), row_bytes bytes (a
@@ -76,13 +182,26 @@ cudaError_t launch_count_positions(const int32_t* idx, long long n, int N, unsig
   return cudaGetLastError();
 }
 
-cudaError_t launch_counts_to_float(unsigned int* counts, int N, cudaStream_t stream) {
-  counts_to_float_kernel<<<(N + 255) / 256, 256, 0, stream>>>(counts, N);
-  return cudaGetLastError();
-}
+size_t rank_scratch_bytes(int n_out) { return 1280 + static_cast<size_t>(n_out) * 8; }
 
-cudaError_t launch_float_to_counts(const float* f, int n, int32_t* out, cudaStream_t stream) {
-  float_to_counts_kernel<<<(n + 255) / 256, 256, 0, stream>>>(f, n, out);
+// Ranks the N counts and writes the n_out most frequent positions; scratch: rank_scratch_bytes(n_out) bytes,
+// 256-byte aligned.
+cudaError_t launch_rank_counts(const unsigned int* counts, int N, int n_out, void* scratch, int32_t* out_pos, int32_t* out_count,
+                               cudaStream_t stream) {
+  static_assert(sizeof(RankState) <= 1088, "state block");
+  RankState* st = static_cast<RankState*>(scratch);
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(static_cast<uint8_t*>(scratch) + 1280);
+  cudaError_t e = cudaMemsetAsync(st, 0, sizeof(RankState), stream);
+  if (e != cudaSuccess) return e;
+  int blocks = (N + 256 * 16 - 1) / (256 * 16);
+  if (blocks < 1) blocks = 1;
+  if (blocks > 148 * 4) blocks = 148 * 4;
+  for (int pass = 0; pass < 8; ++pass) rank_pass_kernel<<<blocks, 256, 0, stream>>>(counts, N, st, pass, n_out);
+  rank_collect_kernel<<<blocks, 256, 0, stream>>>(counts, N, st, keys, n_out);
+  const int smem = next_pow2(n_out < 2 ? 2 : n_out) * 8;
+  e = cudaFuncSetAttribute(rank_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  rank_sort_kernel<<<1, 1024, smem, stream>>>(keys, n_out, out_pos, out_count);
   return cudaGetLastError();
 }
 
