@@ -398,6 +398,32 @@ def run_knn(args, rank: int, local_rank: int, world: int):
         "status": {"bits": status[0], "fallback_rows": status[1], "max_survivors_per_row": status[2],
                    "mean_survivors_per_row": status[3] / inp.T, "overflow_rows": status[4]},
     }
+    if args.knn_sweep and world == 1:
+        sweep = []
+        sizes = [n for n in (1 << 20, 2 << 20, 4 << 20, 5 * 1000 * 1000) if n <= inp.N] or [inp.N]
+        for n_sub in sizes:
+            xs = x[:n_sub]
+            for k_sub in (128, 1024, 4096, 8192):
+                oi = torch.empty((inp.T, k_sub), dtype=torch.int32, device="cuda")
+                ws2 = torch.empty(lt.lt_knn_topk_workspace_bytes(inp.T, n_sub, inp.D, k_sub), dtype=torch.uint8, device="cuda")
+                for _ in range(3):
+                    lt.lt_knn_topk(q, xs, k_sub, oi, None, ws2)
+                torch.cuda.synchronize()
+                ts, sc = [], []
+                for _ in range(10):
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                    lt.lt_knn_topk(q, xs, k_sub, oi, None, ws2)
+                    e1.record(stream)
+                    e1.synchronize()
+                    ts.append(e0.elapsed_time(e1))
+                    sc.append(lt.lt_read_phase_ms()[2])
+                st2 = lt.lt_read_status(ws2)
+                sweep.append({"N": n_sub, "topk": k_sub, "ms_per_step": statistics.median(ts), "scan_ms": statistics.median(sc),
+                              "scan_gbs": n_sub * inp.D * 2 / statistics.median(sc) / 1e6, "fallback_rows": st2[1],
+                              "mean_survivors_per_row": st2[3] / inp.T})
+                del ws2, oi
+        line["sweep"] = sweep
     if not args.no_cpu_baseline and world == 1:
         from oracle import knn_topk
 
@@ -437,6 +463,9 @@ def main():
                     help="also time the auxiliary integer ops on this step's top-k result: lt_topk_frequent and "
                          "lt_dsa_union_mask (group 64); adds an 'aux' object to the JSON line")
     ap.add_argument("--knn-corpus", type=int, default=0, help="k-NN workloads: corpus size (default: the workload's)")
+    ap.add_argument("--knn-sweep", action="store_true",
+                    help="k-NN workloads: also time prefixes of the corpus (1M, 2M, 4M, ... vectors) x k in {128, 1024, 4096, 8192} "
+                         "(the grid of the paper's retrieval benchmark) and add the table as 'sweep'")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-unfused", action="store_true")
     ap.add_argument("--unfused-budget-mb", type=int, default=2048, help="score-matrix budget of the unfused GPU baseline")

@@ -52,13 +52,16 @@ constexpr size_t kGenericScratchBudget = size_t(256) << 20;   // dense scores ke
 
 struct Tun {
   int path, cap_mult, sample_mult, segment_tiles, grid, sample_rank;
-  bool sample_mult_given;
+  bool sample_mult_given, cap_mult_given;
 };
 Tun resolve_tunables(const lt_tunables* t) {
-  Tun r{LT_PATH_AUTO, 12, 3, 0, 0, 0, false};
+  Tun r{LT_PATH_AUTO, 12, 3, 0, 0, 0, false, false};
   if (t != nullptr) {
     r.path = t->path;
-    if (t->cap_mult > 0) r.cap_mult = t->cap_mult;
+    if (t->cap_mult > 0) {
+      r.cap_mult = t->cap_mult;
+      r.cap_mult_given = true;
+    }
     if (t->sample_mult > 0) {
       r.sample_mult = t->sample_mult;
       r.sample_mult_given = true;
@@ -141,7 +144,11 @@ Layout make_layout(bool fused, int T, int N, int topk, int causal_offset, const 
     // With the rank scaled to the sampling fraction the sample only has to hold a few dozen of a row's top-k
     // keys: 64 expected ones (k' = 64 prefix / topk, rounded up to whole key tiles) already put the initial
     // gate within a factor 1.7 of the true k/N quantile.  Short contexts then pay for far fewer sampled
-    // scores (65,536 keys, k = 2048: 2,048 instead of 6,144 per row); at 1M keys the paper's 3k stays.
+    // scores (65,536 keys, k = 2048: 2,048 instead of 6,144 per row).  A small k over a long context is the
+    // opposite case: 3k keys hold less than one of the row's top-k, the gate starts orders of magnitude too
+    // loose and the candidate buffers overflow, so the sample is at least 8,192 keys (6 % of a 1M-key scan
+    // at most).
+    if (want < 8192) want = 8192;
     long long enough = (64 * prefix + topk - 1) / topk;
     enough = (enough + kTileKeys - 1) / kTileKeys * kTileKeys;
     if (enough < want) want = enough;
@@ -173,6 +180,8 @@ Layout make_layout(bool fused, int T, int N, int topk, int causal_offset, const 
   L.gather_scale = off;
   off = align_up(off + static_cast<size_t>(gather_rows) * 4);
   long long cap = static_cast<long long>(tun.cap_mult) * topk;
+  // the paper's 12k is sized for k = 2048; a small k leaves no slack for the looser gate a sample can give
+  if (!tun.cap_mult_given && cap < 16384) cap = 16384;
   L.cap = static_cast<int>(cap > N ? N : cap);
   L.cand = off;
   off = align_up(off + static_cast<size_t>(T) * L.cap * 8);

@@ -164,7 +164,8 @@ def test_monotone_scores_overflow_into_exact_fallback():
     # filtered, the candidate buffers overflow and the rows must come back exact from the fallback
     N, T, topk = 8192, 24, 32
     inp = _axis_inputs(np.arange(1, N + 1), T, topk)
-    idx, score, status = run_topk(inp, lt.Tunables(path=lt.LT_PATH_FUSED, cap_mult=4))
+    # (the paper's 3k-key sample and rank-k rule: the default sample would cover this short context entirely)
+    idx, score, status = run_topk(inp, lt.Tunables(path=lt.LT_PATH_FUSED, cap_mult=4, sample_mult=3, sample_rank=-1))
     assert status[0] & lt.LT_STATUS_FALLBACK and status[1] == T and status[4] == T
     for t in range(T):
         p = inp.causal_offset + t

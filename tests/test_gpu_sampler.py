@@ -101,12 +101,13 @@ def test_previous_chunk_sample_tightens_the_gate_and_keeps_every_bit():
     assert sample.max() <= cur.causal_offset  # every sampled position is visible to every row of the next chunk
     assert len(set(sample.tolist()) & set(both.meta["hot_pos"].tolist())) >= topk
 
-    base_idx, base_score, st_default = run_topk(cur, lt.Tunables(path=lt.LT_PATH_FUSED))
+    # reference point: the paper's rule (3k keys, k-th largest sampled score) on a position-strided sample
+    base_idx, base_score, st_default = run_topk(cur, lt.Tunables(path=lt.LT_PATH_FUSED, sample_mult=3, sample_rank=-1))
     idx, score, st = run_sampled(cur, sample, lt.Tunables(path=lt.LT_PATH_FUSED))
     assert st[0] == 0 and st[1] == 0, st
     assert np.array_equal(idx, base_idx) and np.array_equal(score.view(np.uint32), base_score.view(np.uint32))
     assert_matches_oracle(cur, idx, score, list(range(0, T, 9)))
-    # survivors per row: close to topk with the previous chunk's sample, several times topk with the strided sample
+    # survivors per row: close to topk with the previous chunk's sample, several times topk with the strided one
     assert st[3] / T < 1.6 * topk, st
     assert st[3] < 0.5 * st_default[3], (st, st_default)
 
