@@ -116,3 +116,21 @@ def test_full_size_benchmark_shape():
     assert np.all(np.diff(score.astype(np.float64), axis=1) <= 0)
     dumped = np.concatenate([gpu_scores(inp, r, r + 16) for r in range(0, inp.T, 16)])
     check(inp, idx, score, list(range(inp.T)), dumped)
+
+
+def test_random_shapes():
+    rng = np.random.default_rng(2026)
+    for _ in range(10):
+        T = int(rng.integers(1, 150))
+        D = int(rng.choice([64, 128, 320, 768]))
+        N = int(rng.integers(200, 40000))
+        topk = int(rng.integers(1, min(N, 3000) + 1))
+        inp = make_knn(T=T, N=N, D=D, topk=topk)
+        idx, score, st = gpu_topk(inp)
+        assert st[0] & lt.LT_STATUS_TIMEOUT == 0, (T, N, D, topk)
+        dumped = gpu_scores(inp, 0, T)
+        rows = sorted(set(int(r) for r in rng.integers(0, T, size=3)))
+        check(inp, idx, score, rows, dumped)
+        for t in range(T):
+            want_idx, want_val = canonical_topk_of(dumped[t], inp.N, inp.topk)
+            assert np.array_equal(idx[t].astype(np.int64), want_idx), (T, N, D, topk, t)

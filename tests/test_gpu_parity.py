@@ -239,3 +239,20 @@ def test_adversarial_reduced(name, topk):
         ora = oracle_topk(inp)
         assert np.array_equal(idx.astype(np.int64), ora.idx)
         assert np.array_equal(score.astype(np.float64), ora.score)
+
+
+def test_random_shapes_fused_path():
+    """Seeded random (T, N, topk, causal offset) on both tensor-core dtypes: own-scores rule on every row, oracle on a few."""
+    rng = np.random.default_rng(77)
+    for i in range(10):
+        name = ["dsa_bf16", "fp8_ar1", "hot_fp8", "adv_ties"][i % 4]
+        T = int(rng.integers(1, 100))
+        N = int(rng.integers(T + 64, 30000))
+        topk = int(rng.integers(1, min(N - T, 2500) + 1))
+        inp = make_config(name, T=T, N=N, topk=topk)
+        idx, score, status = run_topk(inp, lt.Tunables(path=lt.LT_PATH_FUSED))
+        assert status[0] & lt.LT_STATUS_TIMEOUT == 0, (name, T, N, topk)
+        dumped = dump_scores(inp, 0, T, lt.LT_PATH_FUSED)
+        rows = sorted(set(int(r) for r in rng.integers(0, T, size=3)))
+        assert_matches_oracle(inp, idx, score, rows, dumped, 0)
+        assert_own_scores_rule(inp, idx, score, dumped, range(T))
