@@ -393,7 +393,7 @@ def run_knn(args, rank: int, local_rank: int, world: int):
                      "kernel_ms": scan_ms, "algorithmic_bytes": alg_bytes,
                      # dram__bytes_read.sum + dram__bytes_write.sum of one launch at the default shape
                      # (profiles/knn_scan_kernel_T64_N1M_D768.md)
-                     "traffic": 1.630325e9 + 45.37e6 if (inp.T, inp.N, inp.D) == (64, 1 << 20, 768) else None},
+                     "traffic": 1.613026e9 + 11.56e6 if (inp.T, inp.N, inp.D) == (64, 1 << 20, 768) else None},
         "phases_ms": {n: statistics.mean(p[i] for p in phase_ms) for i, n in enumerate(names)},
         "status": {"bits": status[0], "fallback_rows": status[1], "max_survivors_per_row": status[2],
                    "mean_survivors_per_row": status[3] / inp.T, "overflow_rows": status[4]},

@@ -121,25 +121,29 @@ __device__ __noinline__ void knn_flush(const uint4* list, int count, const KnnSc
   __syncwarp();
 }
 
-// Appends the survivors of 32 queries (bit q of `mine`: this lane's vector survives query q; bit q of `any`: some
-// lane's does).  Returns the new list length.
-__device__ __forceinline__ int knn_stage32(uint32_t any, uint32_t mine, const uint32_t (&v)[32], int s, int t_first, int lane,
-                                           uint4* list, int count, const KnnScanParams& p, int t0, const float* smin,
-                                           const float* width, const float* inv_width) {
-#pragma unroll
-  for (int q = 0; q < 32; ++q) {
-    if ((any >> q) & 1u) {
-      const bool pass = (mine >> q) & 1u;
-      const uint32_t bal = __ballot_sync(0xffffffffu, pass);
-      if (count + 32 > kKnnStageLen) {
-        knn_flush(list, count, p, t0, smin, width, inv_width);
-        count = 0;
-      }
-      // + 0 turns -0 into +0, so that the bit order of the scores is their value order
-      if (pass) list[count + __popc(bal & ((1u << lane) - 1u))] =
-          make_uint4(__float_as_uint(__fadd_rn(__uint_as_float(v[q]), 0.f)), static_cast<uint32_t>(s), static_cast<uint32_t>(t_first + q), 0u);
-      count += __popc(bal);
+// Appends the survivors of one tile.  mine: bit q set if this lane's vector survives query q; any: bit q set if
+// some lane's does (a handful of bits per tile).  The loop runs over the set bits only and fetches the score of
+// query q again from the tile's accumulator (one TMEM column), which keeps it a few dozen instructions long: a
+// version unrolled over all 64 queries, taking the scores from the registers of the gate, ran out of the
+// instruction cache.  Returns the new list length.
+__device__ __forceinline__ int knn_stage(uint64_t any, uint64_t mine, uint32_t tacc, int s, int lane, uint4* list, int count,
+                                         const KnnScanParams& p, int t0, const float* smin, const float* width,
+                                         const float* inv_width) {
+  while (any != 0ull) {
+    const int q = __ffsll(static_cast<long long>(any)) - 1;
+    any &= any - 1ull;
+    const bool pass = (mine >> q) & 1ull;
+    const uint32_t bal = __ballot_sync(0xffffffffu, pass);
+    const uint32_t x = tmem_ld1(tacc + static_cast<uint32_t>(q));
+    if (count + 32 > kKnnStageLen) {
+      knn_flush(list, count, p, t0, smin, width, inv_width);
+      count = 0;
     }
+    tmem_ld_wait();
+    // + 0 turns -0 into +0, so that the bit order of the scores is their value order
+    if (pass) list[count + __popc(bal & ((1u << lane) - 1u))] =
+        make_uint4(__float_as_uint(__fadd_rn(__uint_as_float(x), 0.f)), static_cast<uint32_t>(s), static_cast<uint32_t>(t0 + q), 0u);
+    count += __popc(bal);
   }
   return count;
 }
@@ -394,10 +398,16 @@ knn_scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           tmem_ld32(tlane + buf * kQB, va);
           tmem_ld32(tlane + buf * kQB + 32, vb);
           tmem_ld_wait();
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&st->bar_acc_empty[buf]));
-          if (!ok) break;
+          if (kMode == kModeDump) {
+            // the dump needs nothing more from the accumulator: hand it back before the stores
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&st->bar_acc_empty[buf]));
+          }
+          if (!ok) {
+            if (kMode == kModeFilter && lane == 0) mbar_arrive(smem_u32(&st->bar_acc_empty[buf]));
+            break;
+          }
           const bool in_range = s < p.n_keys;
           if (kMode == kModeDump) {
 #pragma unroll
@@ -415,8 +425,14 @@ knn_scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const uint32_t mb = knn_gate32(vb, st->thr + 32, in_range);
             const uint32_t any_a = __reduce_or_sync(0xffffffffu, ma);
             const uint32_t any_b = __reduce_or_sync(0xffffffffu, mb);
-            if (any_a != 0u) n_staged = knn_stage32(any_a, ma, va, s, t0, lane, st->stage[ew], n_staged, p, t0, st->smin, st->width, st->inv_width);
-            if (any_b != 0u) n_staged = knn_stage32(any_b, mb, vb, s, t0 + 32, lane, st->stage[ew], n_staged, p, t0, st->smin, st->width, st->inv_width);
+            const uint64_t any = (static_cast<uint64_t>(any_b) << 32) | any_a;
+            if (any != 0ull)
+              n_staged = knn_stage(any, (static_cast<uint64_t>(mb) << 32) | ma, tlane + buf * kQB, s, lane, st->stage[ew], n_staged, p, t0,
+                                   st->smin, st->width, st->inv_width);
+            // the survivors' scores were fetched from the accumulator again: only now hand it back
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&st->bar_acc_empty[buf]));
           }
         }
         if (!ok) dead = true;
