@@ -604,13 +604,15 @@ def main():
         ws = torch.empty(lt.lt_indexer_topk_paged_workspace_bytes(inp.dtype, inp.T, inp.N, inp.H, inp.D, inp.topk),
                          dtype=torch.uint8, device="cuda")
 
-    def step():
+    def step(src=None, dst=None):
+        q_, w_, k_, ks_ = src if src is not None else (q, w, k, ks)
+        idx_, score_ = dst if dst is not None else (out_idx, out_score)
         if page_table is not None:
-            lt.lt_indexer_topk_paged(inp.dtype, q, w, k, ks, page_table, inp.N, inp.topk, inp.causal_offset, out_idx, out_score, ws)
+            lt.lt_indexer_topk_paged(inp.dtype, q_, w_, k_, ks_, page_table, inp.N, inp.topk, inp.causal_offset, idx_, score_, ws)
         elif sample_idx is None:
-            lt.lt_indexer_topk_ex(inp.dtype, q, w, k, ks, inp.topk, inp.causal_offset, out_idx, out_score, ws)
+            lt.lt_indexer_topk_ex(inp.dtype, q_, w_, k_, ks_, inp.topk, inp.causal_offset, idx_, score_, ws)
         else:
-            lt.lt_indexer_topk_sampled(inp.dtype, q, w, k, ks, inp.topk, inp.causal_offset, sample_idx, out_idx, out_score, ws)
+            lt.lt_indexer_topk_sampled(inp.dtype, q_, w_, k_, ks_, inp.topk, inp.causal_offset, sample_idx, idx_, score_, ws)
 
     def barrier():
         if world > 1:
@@ -662,11 +664,55 @@ def main():
 
     e2e_step()
     barrier()
-    e2e_steps = min(args.steps, 5)
+    e2e_steps = min(args.steps, 20)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for _ in range(e2e_steps):
         e2e_step()
+    e1.record(stream)
+    e1.synchronize()
+    e2e_serial_ms = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
+
+    # The same with the copies taken off the compute stream, as a serving loop would run it: two sets of device
+    # input and output buffers, the H2D copy of step i + 1 and the D2H read of step i - 1 on side streams while
+    # step i computes.  Every step still copies all of its inputs in and its results out inside the timed region.
+    h2d_stream, d2h_stream = torch.cuda.Stream(), torch.cuda.Stream()
+    dev2 = [dev, [torch.empty_like(t) for t in dev]]
+    outs2 = [(out_idx, out_score), (torch.empty_like(out_idx), torch.empty_like(out_score))]
+    h_outs2 = [(h_idx, h_score), (torch.empty_like(h_idx).pin_memory(), torch.empty_like(h_score).pin_memory())]
+
+    def e2e_pipelined(n):
+        copied = [torch.cuda.Event() for _ in range(n)]
+        computed = [torch.cuda.Event() for _ in range(n)]
+        read = [torch.cuda.Event() for _ in range(n)]
+        for i in range(n):
+            b = i & 1
+            with torch.cuda.stream(h2d_stream):
+                if i >= 2:
+                    h2d_stream.wait_event(computed[i - 2])  # the step that last read this input set
+                for d, h in zip(dev2[b], host):
+                    d.copy_(h, non_blocking=True)
+                copied[i].record(h2d_stream)
+            stream.wait_event(copied[i])
+            if i >= 2:
+                stream.wait_event(read[i - 2])  # the read that last drained this output set
+            src = tuple(dev2[b]) + ((None,) if ks is None else ())
+            step(src, outs2[b])
+            computed[i].record(stream)
+            with torch.cuda.stream(d2h_stream):
+                d2h_stream.wait_event(computed[i])
+                h_outs2[b][0].copy_(outs2[b][0], non_blocking=True)
+                h_outs2[b][1].copy_(outs2[b][1], non_blocking=True)
+                read[i].record(d2h_stream)
+        for ev in read[-2:]:
+            stream.wait_event(ev)
+
+    e2e_pipelined(2)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    h2d_stream.wait_event(e0)
+    e2e_pipelined(e2e_steps)
     e1.record(stream)
     e1.synchronize()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
@@ -709,7 +755,9 @@ def main():
                    "key_layout": "paged (64-key pages, random order)" if page_table is not None else "dense"},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": e2e_ms / e2e_steps},
+                "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps,
+                "how": "double-buffered: H2D of the next step and D2H of the previous one on side streams",
+                "serial_ms_per_step": e2e_serial_ms / e2e_steps},
         "gpu_launches": int(launches),
         "roofline": roofline,
         "phases_ms": phases,
