@@ -812,12 +812,13 @@ int lt_knn_topk(int dtype, const void* q, const void* x, int T, int N, int D, in
     LT_LAUNCH(launch_final_select(p, stream));
   }
 
-  // 4. exact fallback, one block of 8 rows at a time: dense scores of the block (a launch whose block nobody
+  // 4. exact fallback, as many rows at a time as the scratch holds (the corpus is streamed once per round
+  //    however many rows are scored): dense scores of the round's rows (a launch in whose rows nobody was
   //    flagged returns at once), then the full-row select for the flagged rows
   mark_phase(4, stream);
-  for (int b = 0; b < L.n_blocks; ++b) {
-    const int r0 = b * kRowsPerBlock;
-    const int r1 = r0 + kRowsPerBlock < T ? r0 + kRowsPerBlock : T;
+  const int round_rows = L.fb_slots * kRowsPerBlock;
+  for (int r0 = 0; r0 < T; r0 += round_rows) {
+    const int r1 = r0 + round_rows < T ? r0 + round_rows : T;
     KnnScanParams p{};
     p.T = T;
     p.row_begin = r0;

@@ -77,7 +77,7 @@ struct KnnScanParams {
   // dump mode
   float* dump;             // dense scores, row (t - row_begin)
   long long dump_ld;
-  const unsigned int* fb_flag;  // fallback rounds: flag per block of 8 rows; the launch is a no-op if its block's flag is 0
+  const unsigned int* fb_flag;  // fallback rounds: flag per block of 8 rows; the launch is a no-op if no block of its row range is flagged
   Control* ctl;
 };
 bool scan_knn_supported(int D);

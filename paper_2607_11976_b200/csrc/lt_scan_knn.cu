@@ -163,8 +163,13 @@ knn_scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
 
-  // a fallback round for a row block nobody flagged has nothing to do (uniform across the grid)
-  if (p.fb_flag != nullptr && p.fb_flag[p.row_begin / kRowsPerBlock] == 0u) return;
+  // a fallback round has nothing to do unless some block of 8 rows in [row_begin, row_end) was flagged
+  // (uniform across the grid)
+  if (p.fb_flag != nullptr) {
+    unsigned int any = 0u;
+    for (int b = p.row_begin / kRowsPerBlock; b * kRowsPerBlock < p.row_end; ++b) any |= p.fb_flag[b];
+    if (any == 0u) return;
+  }
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < kKnnStages; ++i) {
