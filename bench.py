@@ -49,6 +49,34 @@ def load_peaks():
     return dict(FALLBACK_PEAKS), "fallback"
 
 
+def time_graph_replay(torch, lt, step, flush, reps: int):
+    """The same step captured once into a CUDA graph and replayed (L2 flushed between replays, untimed): what is
+    left of a step when the host launches nothing.  Phase profiling is off while capturing (event records
+    inside a graph cannot be read back)."""
+    try:
+        lt.lt_set_profiling(False)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step()
+        graph.replay()
+        torch.cuda.synchronize()
+        ms = []
+        for _ in range(reps):
+            if flush is not None:
+                flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            graph.replay()
+            e1.record()
+            e1.synchronize()
+            ms.append(e0.elapsed_time(e1))
+        return {"ms_per_step": statistics.mean(ms), "ms_per_step_min": min(ms), "replays": reps}
+    except Exception as exc:  # noqa: BLE001 - an extra figure, never the headline
+        return {"unavailable": f"{type(exc).__name__}: {exc}"[:160]}
+    finally:
+        lt.lt_set_profiling(True)
+
+
 def measure_fp8_gemm(torch, n: int = 8192, sustained_s: float = 2.0):
     """Dense e4m3 x e4m3 -> bf16 GEMM through the library (cuBLASLt via torch._scaled_mm), measured like the
     bf16 peaks of MEASURED_PEAKS.json: best of 10 single launches (burst) and a back-to-back loop (sustained).
@@ -463,6 +491,8 @@ def run_knn(args, rank: int, local_rank: int, world: int):
                               "mean_survivors_per_row": st2[3] / inp.T})
                 del ws2, oi
         line["sweep"] = sweep
+    if not args.no_graph:
+        line["graph_replay"] = time_graph_replay(torch, lt, step, None, max(args.steps, 20))
     if not args.no_cpu_baseline and world == 1:
         from oracle import knn_topk
 
@@ -507,6 +537,8 @@ def main():
                          "(the grid of the paper's retrieval benchmark) and add the table as 'sweep'")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-unfused", action="store_true")
+    ap.add_argument("--graph", action="store_true", help="indexer workloads: also time the step replayed from a CUDA graph")
+    ap.add_argument("--no-graph", action="store_true", help="k-NN workloads: skip the CUDA-graph replay of the step")
     ap.add_argument("--no-fp8-gemm", action="store_true", help="skip the library FP8 GEMM measured for roofline context")
     ap.add_argument("--unfused-budget-mb", type=int, default=2048, help="score-matrix budget of the unfused GPU baseline")
     args = ap.parse_args()
@@ -797,6 +829,11 @@ def main():
         line["unfused_gpu_baseline"] = {"value": pairs / (ums * 1e-3), "unit": UNIT, "ms_per_step": ums,
                                         "score_buffer_mb": args.unfused_budget_mb}
         del buf
+
+    if args.graph:
+        # off by default here: the step is one 39 ms kernel plus a few small ones, launch overhead is not what it
+        # waits for, and a figure taken this late in the process runs at the lower clocks of a warmed-up GPU
+        line["graph_replay"] = time_graph_replay(torch, lt, step, flush, min(args.steps, 10))
 
     if not args.no_cpu_baseline and world == 1:
         v, rows, npairs, dt = time_oracle(inp, budget_s=args.cpu_budget)
