@@ -32,7 +32,10 @@
  *     which is exact because ReLU is positively homogeneous.
  *   - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work on it
  *     and never synchronise the host, except lt_read_status and the internal
- *     arena growth of the 13-argument lt_indexer_topk.
+ *     arena growth of the 13-argument lt_indexer_topk.  The calls that take a
+ *     workspace can therefore be captured into a CUDA graph (stream capture)
+ *     and replayed, once an eager call of the same kind has loaded the
+ *     kernels; keep lt_set_profiling off while capturing.
  *   - Return value: LT_OK or a negative LT_ERR_* code detected on the host
  *     before anything is enqueued.  Conditions met on the device are recorded
  *     in a status word (LT_STATUS_* bits) inside the workspace; kernels never

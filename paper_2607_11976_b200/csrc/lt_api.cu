@@ -576,8 +576,9 @@ int lt_topk_frequent(const int32_t* idx, int T, int topk, int N, int n_out, int3
   void* scratch = ws + align_up(static_cast<size_t>(N) * 4);
   LT_CUDA(cudaMemsetAsync(counts, 0, static_cast<size_t>(N) * 4, stream));
   LT_LAUNCH(launch_count_positions(idx, static_cast<long long>(T) * topk, N, counts, stream));
-  // rank the N (count, position) pairs with a grid-wide radix select and sort the n_out winners
-  LT_LAUNCH(launch_rank_counts(counts, N, n_out, scratch, out_pos, out_count, stream));
+  // rank the N (count, position) pairs with a grid-wide radix select and order the n_out winners; no position can
+  // occur more often than there are entries
+  LT_LAUNCH(launch_rank_counts(counts, N, n_out, static_cast<unsigned long long>(T) * topk, scratch, out_pos, out_count, stream));
   return LT_OK;
 }
 

@@ -135,10 +135,10 @@ cudaError_t launch_select_rows(const SelectRowsParams& p, cudaStream_t stream);
 // ---- lt_sampler.cu --------------------------------------------------------------------------
 // counts[p] += occurrences of p in idx[0..n) (entries outside [0, N) are skipped); counts must be zeroed.
 cudaError_t launch_count_positions(const int32_t* idx, long long n, int N, unsigned int* counts, cudaStream_t stream);
-// the n_out most frequent positions of counts[0..N), (count desc, position asc); scratch: rank_scratch_bytes(n_out)
+// the n_out most frequent positions of counts[0..N), (count desc, position asc); max_count bounds every count; scratch: rank_scratch_bytes(n_out)
 size_t rank_scratch_bytes(int n_out);
-cudaError_t launch_rank_counts(const unsigned int* counts, int N, int n_out, void* scratch, int32_t* out_pos, int32_t* out_count,
-                               cudaStream_t stream);
+cudaError_t launch_rank_counts(const unsigned int* counts, int N, int n_out, unsigned long long max_count, void* scratch,
+                               int32_t* out_pos, int32_t* out_count, cudaStream_t stream);
 // dense copy of the key rows (row_bytes each, multiple of 16) and scales at the sampled positions (sample_idx, or
 // j * stride when it is null); page_table (or null) translates positions to physical rows of a paged key cache
 cudaError_t launch_gather_keys(const void* k, const float* k_scale, const int32_t* sample_idx, long long stride, int n_sample,
