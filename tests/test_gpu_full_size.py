@@ -95,6 +95,39 @@ def test_full_fp8_1m_paged_cache_gives_the_dense_bits():
     assert abs(st[3] - st0[3]) < 0.01 * st0[3]
 
 
+def test_full_hot_fp8_previous_chunk_sampler_gives_the_same_bits():
+    """Two consecutive 4096-row chunks of one 1M-key context, as `bench.py --workload hot_fp8 --sampler prev_chunk`
+    runs them: the second chunk sampled at the first one's most frequent top-k positions (paper Sec. 3.2
+    "Sampling").  Whatever the sample, the result is the exact top-k of the same scores: identical bits."""
+    import torch
+
+    T = 4096
+    both = make_config("hot_fp8", T=2 * T)
+    n_prev = both.causal_offset + T
+    prev = dataclasses.replace(both, q=both.q[:T], w=both.w[:T], k=both.k[:n_prev], k_scale=both.k_scale[:n_prev])
+    cur = dataclasses.replace(both, q=both.q[T:], w=both.w[T:], causal_offset=both.causal_offset + T)
+    p_idx, _, _ = run_topk(prev)
+    p_idx = torch.from_numpy(p_idx).cuda()
+    n_sample = 3 * prev.topk
+    sample_idx = torch.empty(n_sample, dtype=torch.int32, device="cuda")
+    f_ws = torch.empty(lt.lt_topk_frequent_workspace_bytes(prev.N), dtype=torch.uint8, device="cuda")
+    lt.lt_topk_frequent(p_idx, prev.N, sample_idx, None, f_ws)
+    base_idx, base_score, st0 = run_topk(cur)
+    q, w, k, ks = lt.to_device(cur)
+    out_idx = torch.empty((T, cur.topk), dtype=torch.int32, device="cuda")
+    out_score = torch.empty((T, cur.topk), dtype=torch.float32, device="cuda")
+    ws = torch.empty(lt.lt_indexer_topk_sampled_workspace_bytes(cur.dtype, T, cur.N, cur.H, cur.D, cur.topk, n_sample),
+                     dtype=torch.uint8, device="cuda")
+    lt.lt_indexer_topk_sampled(cur.dtype, q, w, k, ks, cur.topk, cur.causal_offset, sample_idx, out_idx, out_score, ws)
+    st = lt.lt_read_status(ws)
+    assert st[0] & lt.LT_STATUS_TIMEOUT == 0 and st[1] == 0 and st0[1] == 0
+    assert np.array_equal(out_idx.cpu().numpy(), base_idx)
+    assert np.array_equal(out_score.cpu().numpy().view(np.uint32), base_score.view(np.uint32))
+    _check_every_row(cur, base_idx, base_score)
+    # the point of this sampler: its gate starts tighter than the strided sample's rank rule leaves it
+    assert st[3] < st0[3]
+
+
 @pytest.mark.parametrize("name", ["adv_planted", "adv_cluster", "adv_ties", "adv_ties_exact"])
 @pytest.mark.parametrize("topk", [64, 512, 2048, 4096])
 def test_full_adversarial(name, topk):
