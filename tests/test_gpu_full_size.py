@@ -95,6 +95,30 @@ def test_full_fp8_1m_paged_cache_gives_the_dense_bits():
     assert abs(st[3] - st0[3]) < 0.01 * st0[3]
 
 
+def test_full_fp8_1m_result_through_the_integer_ops():
+    """The benchmark's 4096 x 2048 index matrix over 2^20 positions through lt_topk_frequent (3k positions) and
+    lt_dsa_union_mask (groups of 64 rows), the sizes `bench.py --aux` times: every output word against the oracles."""
+    from oracle import frequent_positions, pack_mask_words, union_and_masks
+    from test_gpu_litedsa import gpu_union
+    from test_gpu_sampler import gpu_frequent
+
+    inp = _config("fp8_1m")
+    idx, _, _ = run_topk(inp)
+    n_out = 3 * inp.topk
+    pos, cnt = gpu_frequent(idx, inp.N, n_out)
+    want_pos, want_cnt = frequent_positions(idx.astype(np.int64), inp.N, n_out)
+    assert np.array_equal(pos.astype(np.int64), want_pos) and np.array_equal(cnt.astype(np.int64), want_cnt)
+    group = 64
+    unions, masks = union_and_masks(idx.astype(np.int64), inp.N, group)
+    union_pos, union_len, mask = gpu_union(idx, inp.N, group)
+    words = (group * inp.topk + 31) // 32
+    for g, u in enumerate(unions):
+        assert union_len[g] == u.size and np.array_equal(union_pos[g, :u.size].astype(np.int64), u)
+        assert np.all(union_pos[g, u.size:] == -1)
+    for t in range(0, inp.T, 7):
+        assert np.array_equal(mask[t], pack_mask_words(masks[t], words)), t
+
+
 def test_full_hot_fp8_previous_chunk_sampler_gives_the_same_bits():
     """Two consecutive 4096-row chunks of one 1M-key context, as `bench.py --workload hot_fp8 --sampler prev_chunk`
     runs them: the second chunk sampled at the first one's most frequent top-k positions (paper Sec. 3.2
