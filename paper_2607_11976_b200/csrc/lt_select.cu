@@ -139,15 +139,23 @@ __device__ __forceinline__ uint64_t* radix_sort_by_score_desc(uint64_t* src, uin
   __shared__ unsigned int cnt[kWarps][256];
   __shared__ unsigned int base[256];
   __shared__ int s_skip, s_unsorted;
+  __shared__ unsigned int s_and, s_or;  // bits every score word has / some score word has (known after pass 0)
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int rounds = (n + kRadixThreads - 1) / kRadixThreads;
   const int first = warp * 32 * rounds;
+  if (tid == 0) {
+    s_and = 0xffffffffu;
+    s_or = 0u;
+  }
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 32 + 8 * pass;
+    // a byte that is the same in every score word (usually the leading one) needs no pass at all
+    if (pass > 0 && (((s_and ^ s_or) >> (8 * pass)) & 255u) == 0u) continue;
     for (int i = tid; i < kWarps * 256; i += kRadixThreads) (&cnt[0][0])[i] = 0u;
     __syncthreads();
     uint64_t key[kMaxRounds];
     unsigned int loc[kMaxRounds];
+    unsigned int all_bits = 0xffffffffu, any_bits = 0u;
 #pragma unroll
     for (int r = 0; r < kMaxRounds; ++r) {
       if (r < rounds) {
@@ -163,6 +171,18 @@ __device__ __forceinline__ uint64_t* radix_sort_by_score_desc(uint64_t* src, uin
         if (valid && rank == 0) cnt[warp][d] = before + __popc(peers);
         __syncwarp();
         loc[r] = before + rank;
+        if (valid) {
+          all_bits &= static_cast<unsigned int>(key[r] >> 32);
+          any_bits |= static_cast<unsigned int>(key[r] >> 32);
+        }
+      }
+    }
+    if (pass == 0) {
+      all_bits = __reduce_and_sync(0xffffffffu, all_bits);
+      any_bits = __reduce_or_sync(0xffffffffu, any_bits);
+      if (lane == 0) {
+        atomicAnd(&s_and, all_bits);
+        atomicOr(&s_or, any_bits);
       }
     }
     __syncthreads();
