@@ -382,6 +382,17 @@ __global__ void __launch_bounds__(kFinalThreads) final_select_kernel(const Final
     if (redo) atomicAdd(&p.ctl->overflow_rows, 1);
   }
   if (!redo) {
+    // candidates are fetched eight rounds at a time so that the loads of a batch overlap; the first batch is
+    // issued before the histogram work, which does not depend on it
+    constexpr int kBatch = 8;
+    const uint2* cand = p.cand + static_cast<size_t>(t) * p.cap;
+    const unsigned int rounds = (tail + kFinalThreads - 1) / kFinalThreads;
+    uint2 c[kBatch];
+#pragma unroll
+    for (int j = 0; j < kBatch; ++j) {
+      const unsigned int i = j * kFinalThreads + threadIdx.x;
+      c[j] = (i < tail) ? __ldcs(cand + i) : make_uint2(0xff800000u, 0u);  // -inf never passes a finite edge
+    }
     if (threadIdx.x < kBins) hist[threadIdx.x] = p.hist[static_cast<size_t>(t) * kBins + threadIdx.x];
     if (threadIdx.x == 0) s_count = 0;
     __syncthreads();
@@ -420,16 +431,13 @@ __global__ void __launch_bounds__(kFinalThreads) final_select_kernel(const Final
     }
     __syncthreads();
     const float edge = bin_edge(s_tb, p.smin[t], p.width[t]);
-    const uint2* cand = p.cand + static_cast<size_t>(t) * p.cap;
-    // candidates are fetched eight rounds at a time so that the loads of a batch overlap
-    constexpr int kBatch = 8;
-    const unsigned int rounds = (tail + kFinalThreads - 1) / kFinalThreads;
     for (unsigned int r0 = 0; r0 < rounds; r0 += kBatch) {
-      uint2 c[kBatch];
+      if (r0 > 0) {
 #pragma unroll
-      for (int j = 0; j < kBatch; ++j) {
-        const unsigned int i = (r0 + j) * kFinalThreads + threadIdx.x;
-        c[j] = (i < tail) ? __ldcs(cand + i) : make_uint2(0xff800000u, 0u);  // -inf never passes a finite edge
+        for (int j = 0; j < kBatch; ++j) {
+          const unsigned int i = (r0 + j) * kFinalThreads + threadIdx.x;
+          c[j] = (i < tail) ? __ldcs(cand + i) : make_uint2(0xff800000u, 0u);
+        }
       }
 #pragma unroll
       for (int j = 0; j < kBatch; ++j) {
