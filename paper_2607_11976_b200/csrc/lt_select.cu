@@ -430,34 +430,108 @@ __global__ void __launch_bounds__(kFinalThreads) final_select_kernel(const Final
       if (lane == 0) s_tb = tb;
     }
     __syncthreads();
-    const float edge = bin_edge(s_tb, p.smin[t], p.width[t]);
-    for (unsigned int r0 = 0; r0 < rounds; r0 += kBatch) {
-      if (r0 > 0) {
+    const float smin = p.smin[t], width = p.width[t];
+    const float edge = bin_edge(s_tb, smin, width);
+    // every candidate at or above `from` goes to sel[] (one shared-memory atomic per warp); candidates beyond
+    // sel_cap are counted but not stored
+    auto gather = [&](float from, bool first_batch_loaded) {
+      for (unsigned int r0 = 0; r0 < rounds; r0 += kBatch) {
+        if (r0 > 0 || !first_batch_loaded) {
+#pragma unroll
+          for (int j = 0; j < kBatch; ++j) {
+            const unsigned int i = (r0 + j) * kFinalThreads + threadIdx.x;
+            c[j] = (i < tail) ? __ldcs(cand + i) : make_uint2(0xff800000u, 0u);
+          }
+        }
 #pragma unroll
         for (int j = 0; j < kBatch; ++j) {
           const unsigned int i = (r0 + j) * kFinalThreads + threadIdx.x;
-          c[j] = (i < tail) ? __ldcs(cand + i) : make_uint2(0xff800000u, 0u);
-        }
-      }
-#pragma unroll
-      for (int j = 0; j < kBatch; ++j) {
-        const unsigned int i = (r0 + j) * kFinalThreads + threadIdx.x;
-        const bool take = (i < tail) && (__uint_as_float(c[j].x) >= edge);
-        // one shared-memory atomic per warp
-        const unsigned int ballot = __ballot_sync(0xffffffffu, take);
-        if (ballot != 0) {
-          unsigned int base = 0;
-          if (lane == 0) base = atomicAdd(&s_count, static_cast<unsigned int>(__popc(ballot)));
-          base = __shfl_sync(0xffffffffu, base, 0);
-          if (take) {
-            const unsigned int pos = base + __popc(ballot & ((1u << lane) - 1u));
-            if (pos < static_cast<unsigned int>(sel_cap)) sel[pos] = pack_key(__uint_as_float(c[j].x), static_cast<int>(c[j].y));
+          const bool take = (i < tail) && (__uint_as_float(c[j].x) >= from);
+          const unsigned int ballot = __ballot_sync(0xffffffffu, take);
+          if (ballot != 0) {
+            unsigned int base = 0;
+            if (lane == 0) base = atomicAdd(&s_count, static_cast<unsigned int>(__popc(ballot)));
+            base = __shfl_sync(0xffffffffu, base, 0);
+            if (take) {
+              const unsigned int pos = base + __popc(ballot & ((1u << lane) - 1u));
+              if (pos < static_cast<unsigned int>(sel_cap)) sel[pos] = pack_key(__uint_as_float(c[j].x), static_cast<int>(c[j].y));
+            }
           }
         }
       }
-    }
+    };
+    gather(edge, true);
     __syncthreads();
-    const unsigned int count = s_count;
+    unsigned int count = s_count;
+    if (count > static_cast<unsigned int>(sel_cap) && s_tb >= 1 && s_tb < kBins - 1) {
+      // The threshold bin alone holds more candidates than shared memory takes: equal-width bins over a range that
+      // a few outliers stretch put most keys into a few bins (heavy-tailed scores).  Second level of the same
+      // scheme inside that bin: kBins equal-width bins over [E(tb), E(tb + 1)), the bin in which the count from the
+      // top reaches k, and a second gather from its lower edge.  Costs two more sweeps over the row's candidates
+      // and spares the row the unfused fallback.
+      const int tb = s_tb;
+      const float lo = edge, hi = bin_edge(tb + 1, smin, width);
+      const float w2 = (hi - lo) / static_cast<float>(kBins);
+      if (w2 > 0.f) {
+        __shared__ unsigned int fine[kBins];
+        __shared__ unsigned int s_above;
+        __shared__ float s_from;
+        if (threadIdx.x < kBins) fine[threadIdx.x] = 0u;
+        if (threadIdx.x < 32) {
+          unsigned int above = 0;
+          for (int b = tb + 1 + lane; b < kBins; b += 32) above += hist[b];
+          above = __reduce_add_sync(0xffffffffu, above);
+          if (lane == 0) {
+            s_above = above;
+            s_count = 0;
+          }
+        }
+        __syncthreads();
+        const float inv_w2 = 1.f / w2;
+        for (unsigned int i = threadIdx.x; i < tail; i += kFinalThreads) {
+          const float v = __uint_as_float(__ldg(&cand[i].x));
+          if (v >= lo && v < hi) atomicAdd(&fine[bin_of(v, lo, w2, inv_w2)], 1u);
+        }
+        __syncthreads();
+        if (threadIdx.x < 32) {
+          // the fine bin in which the count from the top (bins above tb included) reaches kk
+          unsigned int cf[8], mine = 0;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            cf[j] = fine[lane * 8 + j];
+            mine += cf[j];
+          }
+          unsigned int incl = mine;
+#pragma unroll
+          for (int d = 1; d < 32; d <<= 1) {
+            const unsigned int o = __shfl_down_sync(0xffffffffu, incl, d);
+            if (lane + d < 32) incl += o;
+          }
+          const unsigned int need = static_cast<unsigned int>(kk) - s_above;  // >= 1: bins above tb hold fewer than kk
+          const unsigned int above = incl - mine;
+          int fb = 0;
+          if (above < need && incl >= need) {
+            unsigned int cum = above;
+            for (int j = 7; j >= 0; --j) {
+              cum += cf[j];
+              if (cum >= need) {
+                fb = lane * 8 + j;
+                break;
+              }
+            }
+          }
+          fb = __reduce_max_sync(0xffffffffu, fb);
+          // fine bin 0 starts at the coarse edge itself: nothing gained, the row is redone
+          if (lane == 0) s_from = fb >= 1 ? fminf(bin_edge(fb, lo, w2), hi) : lo;
+        }
+        __syncthreads();
+        if (s_from > lo) {
+          gather(s_from, false);
+          __syncthreads();
+          count = s_count;
+        }
+      }
+    }
     // count < kk cannot happen for an exact filter; treating it as "redo" keeps the result exact regardless
     if (count > static_cast<unsigned int>(sel_cap) || count < static_cast<unsigned int>(kk)) redo = true;
     if (!redo) {
