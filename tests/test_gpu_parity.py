@@ -187,6 +187,29 @@ def test_decreasing_scores_and_negative_weight_ties():
     assert np.all(score.view(np.uint32) == 0)  # +0.0, never -0.0
 
 
+def test_overfull_threshold_bin_is_rebinned_not_redone():
+    # Scores crowd into one equal-width bin: a few outliers at both ends stretch the sampled range to [0, 254] (bins
+    # one unit wide) while 14,000 keys score between 78.1 and 78.9 in steps of 1/256.  The threshold bin then holds
+    # more candidates than the final select keeps in shared memory; it must re-bin inside that bin, not give up.
+    N, T, topk = 14000, 12, 512
+    rng = np.random.default_rng(5)
+    v = 20000 + rng.integers(0, 200, size=N)
+    # the outliers sit on sampled positions (the strided sample the library will take), so they set the bin range
+    n_sample, stride, _ = lt.lt_indexer_sample_plan(N, topk, N - T)
+    sampled = stride * rng.choice(n_sample, size=46, replace=False)
+    v[sampled[:6]] = 65000
+    v[sampled[6:]] = 1
+    inp = _axis_inputs(v, T, topk)
+    idx, score, status = run_topk(inp, lt.Tunables(path=lt.LT_PATH_FUSED))
+    assert status[1] == 0 and status[0] & lt.LT_STATUS_FALLBACK == 0, "the rows must not need the unfused fallback"
+    assert status[2] > 8192, "the case must overfill the final select's buffer, or it tests nothing"
+    for t in range(T):
+        vis = inp.causal_offset + t + 1
+        order = np.lexsort((np.arange(vis), -v[:vis]))[:topk]  # score descending, index ascending
+        assert idx[t].tolist() == order.tolist()
+        assert score[t].tolist() == (v[order] / 256.0).tolist()
+
+
 def test_forced_overflow_matches_default_bits():
     inp = make_config("dsa_bf16", T=40, N=12000, topk=256)
     base_idx, base_score, st0 = run_topk(inp, lt.Tunables(path=lt.LT_PATH_FUSED))
