@@ -212,13 +212,14 @@ int pick_seg_tiles(const Tun& tun, int n_keys, int n_blocks, int grid) {
   int seg = 256;
   while (seg > 16 && static_cast<long long>(n_blocks) * ((n_tiles + seg - 1) / seg) < 2ll * grid) seg >>= 1;
   // Work items are dealt to the persistent CTAs round-robin, so the launch lasts as long as the CTA with the
-  // most items: among the sizes down to half of the one above, take the shortest such critical path (in key
-  // tiles, plus a few tiles' worth of per-item start-up).  Matters for short chunks: 128 rows over 8192 tiles
-  // are 512 items of 256 tiles (4 rounds on 148 CTAs, the last one half empty) or 592 items of 222 tiles.
+  // most items: among the sizes from the one above down to 16 tiles, take the shortest such critical path (in key
+  // tiles, plus a few tiles' worth of per-item start-up: the query block of an item is as large as four key tiles).
+  // Matters for short chunks: 128 rows over 8192 tiles are 512 items of 256 tiles (4 rounds on 148 CTAs, the last
+  // one half empty) or 592 items of 222 tiles.
   constexpr int kItemOverheadTiles = 4;
   long long best_cost = -1;
   int best = seg;
-  for (int s = seg; s > seg / 2 && s >= 16; --s) {
+  for (int s = seg; s >= 16; --s) {
     const long long items = static_cast<long long>(n_blocks) * ((n_tiles + s - 1) / s);
     const long long rounds = (items + grid - 1) / grid;
     const long long cost = rounds * ((s < n_tiles ? s : n_tiles) + kItemOverheadTiles);
