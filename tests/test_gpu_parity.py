@@ -279,3 +279,15 @@ def test_random_shapes_fused_path():
         rows = sorted(set(int(r) for r in rng.integers(0, T, size=3)))
         assert_matches_oracle(inp, idx, score, rows, dumped, 0)
         assert_own_scores_rule(inp, idx, score, dumped, range(T))
+
+
+@pytest.mark.parametrize("name", ["dsa_bf16", "fp8_ar1", "adv_ties_exact"])
+def test_final_select_branches(name):
+    """Output sizes on both sides of the final select's branch points (radix sort of 512 .. 4096 gathered candidates,
+    select + bitonic sort beyond, tie rows): every row must be the top-k of the library's own scores, in order."""
+    for topk in (300, 511, 512, 2047, 3000, 4095, 4096, 5000):
+        inp = make_config(name, T=12, N=40000, topk=topk)
+        idx, score, status = run_topk(inp, lt.Tunables(path=lt.LT_PATH_FUSED))
+        assert status[0] & lt.LT_STATUS_TIMEOUT == 0, (name, topk)
+        dumped = dump_scores(inp, 0, inp.T, lt.LT_PATH_FUSED)
+        assert_own_scores_rule(inp, idx, score, dumped, range(inp.T))
