@@ -282,10 +282,12 @@ constexpr int kKeepPerThread = 8;  // keys a thread holds in registers per compa
 __device__ __forceinline__ void keep_top_keys(uint64_t* sel, int count, int keep, unsigned int* hist, unsigned int* scratch) {
   __shared__ uint64_t s_prefix64;
   __shared__ unsigned int s_need;
+  __shared__ int s_settled;
   const int tid = threadIdx.x, lane = tid & 31, nthreads = blockDim.x;
   if (tid == 0) {
     s_prefix64 = 0;
     s_need = static_cast<unsigned int>(keep);
+    s_settled = 0;
   }
   uint64_t mask = 0;
   for (int pass = 0; pass < 8; ++pass) {
@@ -319,6 +321,9 @@ __device__ __forceinline__ void keep_top_keys(uint64_t* sel, int count, int keep
           if (cum + c[j] >= need) {
             s_prefix64 = prefix | (static_cast<uint64_t>(lane * 8 + j) << shift);
             s_need = need - cum;
+            // every key with this prefix is wanted: the prefix padded with zeros already separates kept from
+            // dropped keys, the remaining digits need no pass (the usual case once the score bytes are through)
+            if (c[j] == need - cum) s_settled = 1;
             break;
           }
           cum += c[j];
@@ -327,8 +332,9 @@ __device__ __forceinline__ void keep_top_keys(uint64_t* sel, int count, int keep
     }
     mask |= 0xffull << shift;
     __syncthreads();
+    if (s_settled) break;
   }
-  const uint64_t kth = s_prefix64;  // the keep-th largest key itself
+  const uint64_t kth = s_prefix64;  // the keep-th largest key, or a lower bound of it that no dropped key reaches
   // compaction in place, a slab of kKeepPerThread * nthreads keys at a time: every thread pulls its keys of
   // the slab into registers, then the kept ones are written from the front (never past what has been read)
   if (tid == 0) *scratch = 0;
