@@ -85,8 +85,8 @@ extern "C" {
  */
 typedef struct lt_tunables {
   int path;          /* LT_PATH_*                                                        */
-  int cap_mult;      /* candidate buffer capacity per row = cap_mult * topk (the paper's "conservative
-                        capacity 12k", Sec. 4.2).  Default (0): max(12 topk, 16384) entries; an explicit
+  int cap_mult;      /* candidate buffer capacity per row = cap_mult * topk (12 k per row is the size
+                        the paper reports in Sec. 4.2).  Default (0): max(12 topk, 16384) entries; an explicit
                         value is taken as given                                               */
   int sample_mult;   /* sample size k' = sample_mult * topk (paper Sec. 3.2: 3).  Default (0): max(3 topk,
                         8192), but no more than 64 * (keys the sample is drawn from) / topk, which is
@@ -101,14 +101,28 @@ typedef struct lt_tunables {
                         select (fewer than topk survivors) and redone by the exact fallback.
                         -1: r = topk, the paper's rule (Sec. 3.2 "Sampling"), which can never
                         misjudge but starts ~k'/r times looser.  > 0: r itself.              */
-  int reserved[2];
+  int wait_limit_us; /* bound, in microseconds, of every device-side wait of the scan kernels (default 0 = 2 s).
+                        A wait that runs out sets LT_STATUS_TIMEOUT, the kernel unwinds and returns; the
+                        results of that call are invalid, the next call is unaffected               */
+  int debug_flags;   /* LT_DEBUG_* test hooks, 0 in production                             */
 } lt_tunables;
+
+/* lt_tunables.debug_flags (no counterpart in the paper; used by the library's own tests) */
+#define LT_DEBUG_SKIP_ONE_KTILE 1 /* the fused scan's first CTA never loads its first key tile: with a short
+                                     wait_limit_us this exercises the bounded-wait timeout path without
+                                     any fault (the call returns, status has LT_STATUS_TIMEOUT)        */
 
 /*
  * Fused indexer top-k (paper Sec. 3.2; Eq. 1 + Eq. 2), 13-argument form.
  *   dtype is inferred: k_scale != NULL -> q, k are e4m3 codes; k_scale == NULL -> bf16.
- *   out_score may be NULL.  Uses a library-owned workspace that grows on demand
- *   (growth synchronises the device once); lt_shutdown frees it.
+ *   out_score may be NULL.  Uses a library-owned workspace, one per device, that grows on demand
+ *   (growth waits for that device's earlier work once, then frees and reallocates); lt_shutdown
+ *   frees them all.
+ *   All calls of this form on one device share that workspace (counters, histograms, candidate
+ *   buffers, fallback scratch), and each call clears the parts that must start at zero: two calls whose
+ *   kernels may overlap on the GPU (different streams, or different host threads on different
+ *   streams) race on it and return wrong results without any error - serialise them on one stream,
+ *   or use lt_indexer_topk_ex with one workspace per stream.
  */
 int lt_indexer_topk(const void* q, const float* w, const void* k, const float* k_scale,
                     int T, int N, int H, int D, int topk, int causal_offset,
@@ -124,6 +138,18 @@ int lt_indexer_topk_ex(int dtype, const void* q, const float* w, const void* k, 
                        int T, int N, int H, int D, int topk, int causal_offset,
                        int32_t* out_idx, float* out_score,
                        void* workspace, size_t workspace_bytes, const lt_tunables* tunables, void* stream);
+
+/*
+ * lt_indexer_topk_ex over a key matrix whose rows are k_pitch_elems elements apart (k_pitch_elems >= D,
+ * the pitch a multiple of 16 bytes): a view of a wider cache, e.g. one D-wide field of a row that also
+ * holds other data (paper Sec. 4.1 benchmarks the kernel on a serving engine's cache layout).  k_scale
+ * stays dense, one float per key.  Same outputs as the dense layout, bit for bit; same workspace size;
+ * fused tensor-core path only (LT_ERR_UNSUPPORTED otherwise).
+ */
+int lt_indexer_topk_strided(int dtype, const void* q, const float* w, const void* k, long long k_pitch_elems,
+                            const float* k_scale, int T, int N, int H, int D, int topk, int causal_offset,
+                            int32_t* out_idx, float* out_score,
+                            void* workspace, size_t workspace_bytes, const lt_tunables* tunables, void* stream);
 
 /* Bytes of workspace lt_indexer_topk_ex needs for this problem (0 on invalid arguments). */
 size_t lt_indexer_topk_workspace_bytes(int dtype, int T, int N, int H, int D, int topk,
@@ -288,8 +314,8 @@ int lt_unfused_topk(int dtype, const void* q, const float* w, const void* k, con
  *     clears the status block it needs at zero and overwrites score rows before reading them):
  *     two calls whose kernels may overlap on the GPU (different streams, or different host threads
  *     on different streams) race on it - serialise them on one stream;
- *   - the status block is not readable through lt_read_status; device-side waits are bounded as in
- *     every other entry point.
+ *   - the status block lives in the fixed array too: read it with lt_read_status_static; device-side
+ *     waits are bounded as in every other entry point.
  */
 #define LT_STATIC_SCRATCH_BYTES (16u << 20)
 int lt_indexer_topk_static(int dtype, const void* q, const float* w, const void* k, const float* k_scale,
@@ -304,6 +330,16 @@ int lt_indexer_topk_static(int dtype, const void* q, const float* w, const void*
  * workspace == NULL reads the library-owned workspace of lt_indexer_topk.
  */
 int lt_read_status(const void* workspace, int* status8_host, void* stream);
+/* The same for the status block lt_indexer_topk_static keeps in the current device's fixed array. */
+int lt_read_status_static(int* status8_host, void* stream);
+
+/*
+ * Test probe for the bounded waits (no counterpart in the paper): one warp waits, with the wait
+ * every scan kernel uses, at most limit_us microseconds on a barrier nobody arrives at.  On return of
+ * the kernel result2_device[0] = 0 (the wait gave up) and result2_device[1] = 1 (it raised the abort
+ * flag its CTA would unwind on).  Nothing faults, traps or spins without bound.
+ */
+int lt_debug_wait_timeout(int limit_us, int* result2_device, void* stream);
 
 /*
  * Instrumentation (no counterpart in the paper; used by the benchmark).

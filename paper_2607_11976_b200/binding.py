@@ -19,6 +19,7 @@ LT_DTYPE_F32, LT_DTYPE_BF16, LT_DTYPE_E4M3 = 0, 1, 2
 LT_PATH_AUTO, LT_PATH_FUSED, LT_PATH_GENERIC = 0, 1, 2
 LT_OK = 0
 LT_STATUS_TIMEOUT, LT_STATUS_FALLBACK, LT_STATUS_BOUNDS = 1, 2, 4
+LT_DEBUG_SKIP_ONE_KTILE = 1
 LT_MAX_TOPK = 8192
 
 _DTYPE_CODES = {"f32": LT_DTYPE_F32, "bf16": LT_DTYPE_BF16, "e4m3": LT_DTYPE_E4M3}
@@ -35,14 +36,23 @@ class Tunables(ctypes.Structure):
 
     _fields_ = [("path", ctypes.c_int), ("cap_mult", ctypes.c_int), ("sample_mult", ctypes.c_int),
                 ("segment_tiles", ctypes.c_int), ("grid", ctypes.c_int), ("sample_rank", ctypes.c_int),
-                ("reserved", ctypes.c_int * 2)]
+                ("wait_limit_us", ctypes.c_int), ("debug_flags", ctypes.c_int)]
 
 
 _lib = None
+_lib_path = None
 
 
 def library_path() -> str:
-    return _build.LIB_PATH
+    return _lib_path or _build.LIB_PATH
+
+
+def use_library(path: Optional[str]) -> None:
+    """Selects which build of the library `load()` opens (None: the release build).  Used by the tests
+    that run the bounds-checking build (`build.build(debug_bounds=True)`)."""
+    global _lib, _lib_path
+    _lib_path = path
+    _lib = None
 
 
 def load() -> ctypes.CDLL:
@@ -93,6 +103,13 @@ def load() -> ctypes.CDLL:
     lib.lt_indexer_topk_static.restype = i
     lib.lt_read_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int), vp]
     lib.lt_read_status.restype = i
+    lib.lt_read_status_static.argtypes = [ctypes.POINTER(ctypes.c_int), vp]
+    lib.lt_read_status_static.restype = i
+    lib.lt_debug_wait_timeout.argtypes = [i, ip, vp]
+    lib.lt_debug_wait_timeout.restype = i
+    lib.lt_indexer_topk_strided.argtypes = [i, vp, fp, vp, ctypes.c_longlong, fp, i, i, i, i, i, i, ip, fp, vp, sz,
+                                            ctypes.POINTER(Tunables), vp]
+    lib.lt_indexer_topk_strided.restype = i
     lib.lt_launch_count.restype = ctypes.c_ulonglong
     lib.lt_set_profiling.argtypes = [i]
     lib.lt_set_profiling.restype = i
@@ -170,6 +187,22 @@ def lt_indexer_topk_ex(dtype, q, w, k, k_scale, topk: int, causal_offset: int, o
                                      causal_offset, _ptr(out_idx), _ptr(out_score), _ptr(workspace),
                                      workspace.numel() * workspace.element_size(),
                                      ctypes.byref(tunables) if tunables else None, _stream(stream)), "lt_indexer_topk_ex")
+
+
+def lt_indexer_topk_strided(dtype, q, w, k_view, k_scale, topk: int, causal_offset: int, out_idx, out_score, workspace,
+                            tunables: Optional[Tunables] = None, stream=None) -> None:
+    """lt_indexer_topk_ex over a row-strided key view: `k_view` is an [N, D] CUDA tensor whose rows are
+    `k_view.stride(0)` elements apart (inner stride 1), e.g. `cache[:, :D]` of a wider cache."""
+    T, H, D = q.shape
+    N, D2 = k_view.shape
+    if D2 != D or k_view.stride(1) != 1 or not k_view.is_cuda:
+        raise ValueError("expected an [N, D] CUDA view with unit inner stride")
+    _check(load().lt_indexer_topk_strided(dtype_code(dtype), _ptr(q), _ptr(w), ctypes.c_void_p(k_view.data_ptr()),
+                                          int(k_view.stride(0)), _ptr(k_scale), T, N, H, D, topk, causal_offset,
+                                          _ptr(out_idx), _ptr(out_score), _ptr(workspace),
+                                          workspace.numel() * workspace.element_size(),
+                                          ctypes.byref(tunables) if tunables else None, _stream(stream)),
+           "lt_indexer_topk_strided")
 
 
 def lt_indexer_topk_sampled_workspace_bytes(dtype, T: int, N: int, H: int, D: int, topk: int, n_sample: int,
@@ -278,6 +311,18 @@ def lt_read_status(workspace=None, stream=None) -> list:
     buf = (ctypes.c_int * 8)()
     _check(load().lt_read_status(_ptr(workspace), buf, _stream(stream)), "lt_read_status")
     return list(buf)
+
+
+def lt_read_status_static(stream=None) -> list:
+    """The status block of the last lt_indexer_topk_static call on the current device."""
+    buf = (ctypes.c_int * 8)()
+    _check(load().lt_read_status_static(buf, _stream(stream)), "lt_read_status_static")
+    return list(buf)
+
+
+def lt_debug_wait_timeout(limit_us: int, result2, stream=None) -> None:
+    """Runs the bounded-wait probe: result2 (int32 CUDA tensor of 2) receives (wait result, abort flag)."""
+    _check(load().lt_debug_wait_timeout(int(limit_us), _ptr(result2), _stream(stream)), "lt_debug_wait_timeout")
 
 
 def lt_launch_count() -> int:

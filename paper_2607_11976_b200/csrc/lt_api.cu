@@ -53,9 +53,11 @@ constexpr size_t kGenericScratchBudget = size_t(256) << 20;   // dense scores ke
 struct Tun {
   int path, cap_mult, sample_mult, segment_tiles, grid, sample_rank;
   bool sample_mult_given, cap_mult_given;
+  unsigned int wait_limit_us;
+  int debug_flags;
 };
 Tun resolve_tunables(const lt_tunables* t) {
-  Tun r{LT_PATH_AUTO, 12, 3, 0, 0, 0, false, false};
+  Tun r{LT_PATH_AUTO, 12, 3, 0, 0, 0, false, false, 0u, 0};
   if (t != nullptr) {
     r.path = t->path;
     if (t->cap_mult > 0) {
@@ -69,6 +71,8 @@ Tun resolve_tunables(const lt_tunables* t) {
     if (t->segment_tiles > 0) r.segment_tiles = t->segment_tiles;
     if (t->grid > 0) r.grid = t->grid;
     r.sample_rank = t->sample_rank;
+    if (t->wait_limit_us > 0) r.wait_limit_us = static_cast<unsigned int>(t->wait_limit_us);
+    r.debug_flags = t->debug_flags;
   }
   return r;
 }
@@ -243,6 +247,7 @@ int run_unfused(int dtype, bool mma, const void* q, const float* w, const void* 
     const int r1 = (r0 + rows_per_pass < T) ? r0 + rows_per_pass : T;
     if (mma) {
       ScanParams p{};
+      p.wait_limit_us = tun.wait_limit_us;
       p.w = w;
       p.k_scale = k_scale;
       p.ks_stride = 1;
@@ -285,9 +290,11 @@ size_t elem_bytes(int dtype) { return dtype == LT_DTYPE_F32 ? 4 : (dtype == LT_D
 int topk_impl(int dtype, const void* q, const float* w, const void* k, const float* k_scale, int T, int N, int H, int D, int topk,
               int causal_offset, int32_t* out_idx, float* out_score, void* workspace, size_t workspace_bytes,
               const lt_tunables* tunables, cudaStream_t stream, const int32_t* sample_idx = nullptr, int n_given = 0,
-              const int* page_table = nullptr, int n_pages = 0, long long pool_rows = 0) {
+              const int* page_table = nullptr, int n_pages = 0, long long pool_rows = 0, long long key_pitch_elems = 0) {
   int rc = check_problem(dtype, q, w, k, k_scale, T, N, H, D);
   if (rc != LT_OK) return rc;
+  // distance between consecutive key rows in elements (a strided view of a wider cache); dense by default
+  const long long key_pitch = key_pitch_elems > 0 ? key_pitch_elems : D;
   if (out_idx == nullptr || topk <= 0 || topk > N || topk > LT_MAX_TOPK) return LT_ERR_INVALID_ARG;
   const Tun tun = resolve_tunables(tunables);
   const bool fused = use_fused(tun, dtype, H, D);
@@ -295,6 +302,7 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
   const int key_row_bytes = static_cast<int>(static_cast<size_t>(D) * elem_bytes(dtype));
   const bool paged = page_table != nullptr;
   if (paged && !fused) return LT_ERR_UNSUPPORTED;
+  if (key_pitch != D && (!fused || paged || n_given > 0)) return LT_ERR_UNSUPPORTED;
   const Layout L = make_layout(fused, T, N, topk, causal_offset, tun, n_given, key_row_bytes, paged);
   const long long key_rows = paged ? pool_rows : N;  // rows the key tensor map covers
   if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) != 0 || workspace_bytes < L.total)
@@ -326,11 +334,12 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
   mark_phase(0, stream);
   const void* sample_keys = k;
   const float* sample_scale = k_scale;
-  long long sample_pitch = static_cast<long long>(L.sample_stride) * D;
+  long long sample_pitch = static_cast<long long>(L.sample_stride) * key_pitch;
   long long sample_ks_stride = L.sample_stride;
   if ((n_given > 0 || paged) && L.n_sample > 0) {
     LT_LAUNCH(launch_gather_keys(k, k_scale, n_given > 0 ? sample_idx : nullptr, L.sample_stride, L.n_sample, N, key_row_bytes,
-                                 page_table, ws + L.gather_k, reinterpret_cast<float*>(ws + L.gather_scale), stream));
+                                 page_table, pool_rows, ctl, ws + L.gather_k, reinterpret_cast<float*>(ws + L.gather_scale),
+                                 stream));
     sample_keys = ws + L.gather_k;
     if (k_scale != nullptr) sample_scale = reinterpret_cast<const float*>(ws + L.gather_scale);
     sample_pitch = D;
@@ -338,6 +347,7 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
   }
   if (L.n_sample > 0) {
     ScanParams p{};
+    p.wait_limit_us = tun.wait_limit_us;
     p.w = w;
     p.k_scale = sample_scale;
     p.ks_stride = sample_ks_stride;
@@ -361,6 +371,7 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
   // 2. fused scan: score, gate, compact, count
   {
     ScanParams p{};
+    p.wait_limit_us = tun.wait_limit_us;
     p.w = w;
     p.k_scale = k_scale;
     p.ks_stride = 1;
@@ -381,8 +392,10 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
     p.cap = L.cap;
     p.page_table = page_table;
     p.n_pages = n_pages;
+    p.pool_pages = pool_rows / kPageKeys;
+    p.debug_flags = tun.debug_flags;
     p.ctl = ctl;
-    LT_LAUNCH(launch_scan_mma(dtype, kModeFilter, q, T, k, key_rows, D, p, grid, stream));
+    LT_LAUNCH(launch_scan_mma(dtype, kModeFilter, q, T, k, key_rows, key_pitch, p, grid, stream));
   }
 
   // 3. final select over the survivors; rows it cannot finish exactly are flagged
@@ -414,6 +427,7 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
   const int rounds = (L.n_blocks + L.fb_slots - 1) / L.fb_slots;
   for (int r = 0; r < rounds; ++r) {
     ScanParams p{};
+    p.wait_limit_us = tun.wait_limit_us;
     p.w = w;
     p.k_scale = k_scale;
     p.ks_stride = 1;
@@ -433,8 +447,9 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
     p.fb_slots = L.fb_slots;
     p.page_table = page_table;
     p.n_pages = n_pages;
+    p.pool_pages = pool_rows / kPageKeys;
     p.ctl = ctl;
-    LT_LAUNCH(launch_scan_mma(dtype, kModeDump, q, T, k, key_rows, D, p, grid, stream));
+    LT_LAUNCH(launch_scan_mma(dtype, kModeDump, q, T, k, key_rows, key_pitch, p, grid, stream));
     SelectRowsParams sp{};
     sp.scores = scratch;
     sp.ld = N;
@@ -482,10 +497,11 @@ int static_scratch_address(void** out) {
 }
 
 // ---- library-owned workspace of the 13-argument entry point -----------------------------------
+// One arena per device, grown on demand; g_arena_mu is held while a call's work is enqueued.
+constexpr int kMaxDevices = 64;
 std::mutex g_arena_mu;
-void* g_arena = nullptr;
-size_t g_arena_bytes = 0;
-int g_arena_dev = -1;
+void* g_arena[kMaxDevices] = {nullptr};
+size_t g_arena_bytes[kMaxDevices] = {0};
 
 }  // namespace
 }  // namespace lt
@@ -608,6 +624,17 @@ int lt_indexer_topk_ex(int dtype, const void* q, const float* w, const void* k, 
                    tunables, static_cast<cudaStream_t>(stream));
 }
 
+int lt_indexer_topk_strided(int dtype, const void* q, const float* w, const void* k, long long k_pitch_elems,
+                            const float* k_scale, int T, int N, int H, int D, int topk, int causal_offset, int32_t* out_idx,
+                            float* out_score, void* workspace, size_t workspace_bytes, const lt_tunables* tunables,
+                            void* stream) {
+  if (k_pitch_elems < D) return LT_ERR_INVALID_ARG;
+  // the tensor map wants row pitches that are multiples of 16 bytes
+  if ((static_cast<size_t>(k_pitch_elems) * elem_bytes(dtype)) % 16 != 0) return LT_ERR_INVALID_ARG;
+  return topk_impl(dtype, q, w, k, k_scale, T, N, H, D, topk, causal_offset, out_idx, out_score, workspace, workspace_bytes,
+                   tunables, static_cast<cudaStream_t>(stream), nullptr, 0, nullptr, 0, 0, k_pitch_elems);
+}
+
 int lt_indexer_topk(const void* q, const float* w, const void* k, const float* k_scale, int T, int N, int H, int D, int topk,
                     int causal_offset, int32_t* out_idx, float* out_score, void* stream) {
   const int dtype = (k_scale != nullptr) ? LT_DTYPE_E4M3 : LT_DTYPE_BF16;
@@ -619,19 +646,20 @@ int lt_indexer_topk(const void* q, const float* w, const void* k, const float* k
   std::lock_guard<std::mutex> lock(g_arena_mu);
   int dev = 0;
   LT_CUDA(cudaGetDevice(&dev));
-  if (g_arena == nullptr || g_arena_bytes < need || g_arena_dev != dev) {
-    if (g_arena != nullptr) {
+  if (dev < 0 || dev >= kMaxDevices) return LT_ERR_UNSUPPORTED;
+  if (g_arena[dev] == nullptr || g_arena_bytes[dev] < need) {
+    if (g_arena[dev] != nullptr) {
+      // earlier calls on this device may still be using the old arena: wait for them before it is freed
       LT_CUDA(cudaDeviceSynchronize());
-      cudaFree(g_arena);
-      g_arena = nullptr;
-      g_arena_bytes = 0;
+      cudaFree(g_arena[dev]);
+      g_arena[dev] = nullptr;
+      g_arena_bytes[dev] = 0;
     }
-    LT_CUDA(cudaMalloc(&g_arena, need));
-    g_arena_bytes = need;
-    g_arena_dev = dev;
+    LT_CUDA(cudaMalloc(&g_arena[dev], need));
+    g_arena_bytes[dev] = need;
   }
-  return topk_impl(dtype, q, w, k, k_scale, T, N, H, D, topk, causal_offset, out_idx, out_score, g_arena, g_arena_bytes, nullptr,
-                   static_cast<cudaStream_t>(stream));
+  return topk_impl(dtype, q, w, k, k_scale, T, N, H, D, topk, causal_offset, out_idx, out_score, g_arena[dev], g_arena_bytes[dev],
+                   nullptr, static_cast<cudaStream_t>(stream));
 }
 
 int lt_indexer_scores(int dtype, const void* q, const float* w, const void* k, const float* k_scale, int T, int N, int H, int D,
@@ -653,6 +681,7 @@ int lt_indexer_scores(int dtype, const void* q, const float* w, const void* k, c
   if (mma) {
     // the scan kernel addresses dump rows relative to row_begin
     ScanParams p{};
+    p.wait_limit_us = tun.wait_limit_us;
     const int grid = sm_count();
     p.w = w;
     p.k_scale = kk;
@@ -750,11 +779,12 @@ int lt_knn_topk(int dtype, const void* q, const void* x, int T, int N, int D, in
   uint2* cand = reinterpret_cast<uint2*>(ws + L.cand);
   float* scratch = reinterpret_cast<float*>(ws + L.scratch);
 
-  // 1. sample phase (paper Sec. 3.2 "Sampling": "for k-NN search ... random sampling suffices"): a strided
-  //    view of the corpus, scored by the same tensor-core kernel
+  // 1. sample phase (paper Sec. 3.2 "Sampling": k-NN needs no history-based sample; a strided subsample of
+  //    the corpus is used here), scored by the same tensor-core kernel
   mark_phase(0, stream);
   if (L.n_sample > 0) {
     KnnScanParams p{};
+    p.wait_limit_us = tun.wait_limit_us;
     p.T = T;
     p.row_begin = 0;
     p.row_end = T;
@@ -773,6 +803,7 @@ int lt_knn_topk(int dtype, const void* q, const void* x, int T, int N, int D, in
   // 2. fused scan: one pass over the corpus
   {
     KnnScanParams p{};
+    p.wait_limit_us = tun.wait_limit_us;
     p.T = T;
     p.row_begin = 0;
     p.row_end = T;
@@ -822,6 +853,7 @@ int lt_knn_topk(int dtype, const void* q, const void* x, int T, int N, int D, in
   for (int r0 = 0; r0 < T; r0 += round_rows) {
     const int r1 = r0 + round_rows < T ? r0 + round_rows : T;
     KnnScanParams p{};
+    p.wait_limit_us = tun.wait_limit_us;
     p.T = T;
     p.row_begin = r0;
     p.row_end = r1;
@@ -906,11 +938,29 @@ int lt_read_status(const void* workspace, int* status8_host, void* stream) {
   const void* src = workspace;
   if (src == nullptr) {
     std::lock_guard<std::mutex> lock(g_arena_mu);
-    src = g_arena;
+    int dev = 0;
+    LT_CUDA(cudaGetDevice(&dev));
+    if (dev >= 0 && dev < kMaxDevices) src = g_arena[dev];
   }
   if (src == nullptr) return LT_ERR_WORKSPACE;
   LT_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
   LT_CUDA(cudaMemcpy(status8_host, src, 8 * sizeof(int), cudaMemcpyDeviceToHost));
+  return LT_OK;
+}
+
+int lt_read_status_static(int* status8_host, void* stream) {
+  if (status8_host == nullptr) return LT_ERR_INVALID_ARG;
+  void* base = nullptr;
+  int rc = static_scratch_address(&base);
+  if (rc != LT_OK) return rc;
+  LT_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+  LT_CUDA(cudaMemcpy(status8_host, base, 8 * sizeof(int), cudaMemcpyDeviceToHost));
+  return LT_OK;
+}
+
+int lt_debug_wait_timeout(int limit_us, int* result2_device, void* stream) {
+  if (limit_us <= 0 || result2_device == nullptr) return LT_ERR_INVALID_ARG;
+  LT_LAUNCH(launch_wait_timeout_probe(static_cast<unsigned int>(limit_us), result2_device, static_cast<cudaStream_t>(stream)));
   return LT_OK;
 }
 
@@ -943,13 +993,19 @@ int lt_read_phase_ms(float* ms5_host, void* stream) {
 
 void lt_shutdown(void) {
   std::lock_guard<std::mutex> lock(g_arena_mu);
-  if (g_arena != nullptr) {
-    cudaDeviceSynchronize();
-    cudaFree(g_arena);
-    g_arena = nullptr;
-    g_arena_bytes = 0;
-    g_arena_dev = -1;
+  int cur = 0;
+  if (cudaGetDevice(&cur) != cudaSuccess) cur = -1;
+  for (int dev = 0; dev < kMaxDevices; ++dev) {
+    if (g_arena[dev] == nullptr) continue;
+    // the arena belongs to `dev`: make it current, wait for its work, free
+    if (cudaSetDevice(dev) == cudaSuccess) {
+      cudaDeviceSynchronize();
+      cudaFree(g_arena[dev]);
+    }
+    g_arena[dev] = nullptr;
+    g_arena_bytes[dev] = 0;
   }
+  if (cur >= 0) cudaSetDevice(cur);
 }
 
 }  // extern "C"

@@ -25,6 +25,22 @@ struct Control {
 };
 
 // ---------------------------------------------------------------------------------------------
+// Index checks of the bounds-checking build (compiled with -DLT_DEBUG_BOUNDS; it stands in for a memory
+// checker): LT_IN_BOUNDS(cond, ctl) is `cond`, and where it is false it records LT_STATUS_BOUNDS in the
+// status word so that the caller can skip the access and carry on - nothing traps.  In the release build
+// it is the constant true and costs nothing.
+// ---------------------------------------------------------------------------------------------
+#if defined(LT_DEBUG_BOUNDS)
+__device__ __forceinline__ bool lt_in_bounds(bool cond, Control* ctl) {
+  if (!cond && ctl != nullptr) atomicOr(&ctl->status, LT_STATUS_BOUNDS);
+  return cond;
+}
+#define LT_IN_BOUNDS(cond, ctl) (::lt::lt_in_bounds((cond), (ctl)))
+#else
+#define LT_IN_BOUNDS(cond, ctl) (true)
+#endif
+
+// ---------------------------------------------------------------------------------------------
 // total order on (score, index): larger key = better.  Scores are canonicalised (-0 -> +0)
 // where they are produced, so bit order equals value order.
 // ---------------------------------------------------------------------------------------------

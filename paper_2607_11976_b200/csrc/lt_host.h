@@ -46,11 +46,18 @@ struct ScanParams {
   // the pool the key tensor map covers; k_scale is then indexed by physical row
   const int* page_table;
   int n_pages;
+  long long pool_pages;    // pages of the pool behind page_table (bounds checks of the debug build)
+  unsigned int wait_limit_us;  // bound of every device-side wait (0 is replaced by the default at launch)
+  int debug_flags;         // LT_DEBUG_* test hooks (filter mode only)
   Control* ctl;
 };
 constexpr int kPageKeys = 64;  // keys per page of a paged key cache
 
 bool scan_mma_supported(int dtype, int H, int D);
+
+// One warp waits, with the bounded wait every scan kernel uses, on a barrier nobody arrives at:
+// result2[0] = what the wait returned (0 = gave up), result2[1] = the abort flag it left behind.
+cudaError_t launch_wait_timeout_probe(unsigned int limit_us, int* result2, cudaStream_t stream);
 
 // q: [T][64][128]; k: view of n_keys_view rows whose pitch is key_pitch_elems elements.
 cudaError_t launch_scan_mma(int dtype, int mode, const void* q, int T, const void* k, long long n_keys_view,
@@ -78,6 +85,7 @@ struct KnnScanParams {
   float* dump;             // dense scores, row (t - row_begin)
   long long dump_ld;
   const unsigned int* fb_flag;  // fallback rounds: flag per block of 8 rows; the launch is a no-op if no block of its row range is flagged
+  unsigned int wait_limit_us;   // bound of every device-side wait (0 is replaced by the default at launch)
   Control* ctl;
 };
 bool scan_knn_supported(int D);
@@ -141,8 +149,10 @@ cudaError_t launch_rank_counts(const unsigned int* counts, int N, int n_out, uns
                                int32_t* out_pos, int32_t* out_count, cudaStream_t stream);
 // dense copy of the key rows (row_bytes each, multiple of 16) and scales at the sampled positions (sample_idx, or
 // j * stride when it is null); page_table (or null) translates positions to physical rows of a paged key cache
+// (pool_rows and ctl serve the bounds-checking build: a translated row outside the pool is read as row 0 and flagged)
 cudaError_t launch_gather_keys(const void* k, const float* k_scale, const int32_t* sample_idx, long long stride, int n_sample,
-                               int N, int row_bytes, const int* page_table, void* out_k, float* out_scale, cudaStream_t stream);
+                               int N, int row_bytes, const int* page_table, long long pool_rows, Control* ctl, void* out_k,
+                               float* out_scale, cudaStream_t stream);
 
 // ---- lt_dsa_union.cu ------------------------------------------------------------------------
 // LiteDSA union list + membership masks of consecutive groups of `group` rows (paper Sec. 3.3).

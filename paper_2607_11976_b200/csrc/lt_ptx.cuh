@@ -41,11 +41,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait: gives up after `limit_ns` of wall time or as soon as *abort_flag is set by anyone.
-// Returns false on give-up (and sets *abort_flag), so callers can unwind without hanging the GPU.
-constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
+// Bounded wait: gives up after `limit_us` microseconds of wall time or as soon as *abort_flag is set by
+// anyone.  Returns false on give-up (and sets *abort_flag), so callers can unwind without hanging the GPU.
+constexpr uint32_t kDefaultWaitLimitUs = 2000000u;  // 2 s
 template <int kBackoffNs = 0>
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t limit_us) {
   uint64_t t0 = 0;
   for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -55,7 +55,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       uint64_t now = globaltimer_ns();
       if (t0 == 0) {
         t0 = now;
-      } else if (now - t0 > kWaitLimitNs) {
+      } else if (now - t0 > static_cast<uint64_t>(limit_us) * 1000ull) {
         *abort_flag = 1;
         return false;
       }

@@ -199,7 +199,8 @@ __global__ void __launch_bounds__(256) rank_write_kernel(const unsigned long lon
 __global__ void __launch_bounds__(256) gather_keys_kernel(const uint8_t* __restrict__ k, const float* __restrict__ k_scale,
                                                           const int32_t* __restrict__ sample_idx, long long stride,
                                                           int n_sample, int N, int row_bytes,
-                                                          const int* __restrict__ page_table, uint8_t* __restrict__ out_k,
+                                                          const int* __restrict__ page_table, long long pool_rows,
+                                                          Control* ctl, uint8_t* __restrict__ out_k,
                                                           float* __restrict__ out_scale) {
   const int pieces = row_bytes >> 4;
   const long long g = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -208,7 +209,10 @@ __global__ void __launch_bounds__(256) gather_keys_kernel(const uint8_t* __restr
   if (j >= n_sample) return;
   long long s = sample_idx != nullptr ? static_cast<long long>(__ldg(sample_idx + j)) : j * stride;
   if (s < 0 || s >= N) s = 0;
-  if (page_table != nullptr) s = static_cast<long long>(__ldg(page_table + s / kPageKeys)) * kPageKeys + s % kPageKeys;
+  if (page_table != nullptr) {
+    s = static_cast<long long>(__ldg(page_table + s / kPageKeys)) * kPageKeys + s % kPageKeys;
+    if (!LT_IN_BOUNDS(s >= 0 && s < pool_rows, ctl)) s = 0;  // a page-table entry outside the pool
+  }
   const uint4 v = __ldg(reinterpret_cast<const uint4*>(k + static_cast<size_t>(s) * row_bytes) + piece);
   reinterpret_cast<uint4*>(out_k + static_cast<size_t>(j) * row_bytes)[piece] = v;
   if (piece == 0 && k_scale != nullptr) out_scale[j] = __ldg(k_scale + s);
@@ -263,10 +267,11 @@ cudaError_t launch_rank_counts(const unsigned int* counts, int N, int n_out, uns
 }
 
 cudaError_t launch_gather_keys(const void* k, const float* k_scale, const int32_t* sample_idx, long long stride, int n_sample,
-                               int N, int row_bytes, const int* page_table, void* out_k, float* out_scale, cudaStream_t stream) {
+                               int N, int row_bytes, const int* page_table, long long pool_rows, Control* ctl, void* out_k,
+                               float* out_scale, cudaStream_t stream) {
   const long long threads = static_cast<long long>(n_sample) * (row_bytes >> 4);
   gather_keys_kernel<<<static_cast<int>((threads + 255) / 256), 256, 0, stream>>>(
-      static_cast<const uint8_t*>(k), k_scale, sample_idx, stride, n_sample, N, row_bytes, page_table,
+      static_cast<const uint8_t*>(k), k_scale, sample_idx, stride, n_sample, N, row_bytes, page_table, pool_rows, ctl,
       static_cast<uint8_t*>(out_k), out_scale);
   return cudaGetLastError();
 }

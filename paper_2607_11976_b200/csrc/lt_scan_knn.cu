@@ -113,10 +113,12 @@ __device__ __noinline__ void knn_flush(const uint4* list, int count, const KnnSc
   for (int i = lane; i < count; i += 32) {
     const uint4 e = list[i];
     const int t = static_cast<int>(e.z);
+    const int r = t - t0;
+    if (!LT_IN_BOUNDS(t >= 0 && t < p.T && r >= 0 && r < kQB && e.y < static_cast<uint32_t>(p.n_keys), p.ctl)) continue;
     const uint32_t pos = atomicAdd(p.tail + t, 1u);
     if (pos < static_cast<uint32_t>(p.cap)) p.cand[static_cast<size_t>(t) * p.cap + pos] = make_uint2(e.x, e.y);
-    const int r = t - t0;
-    atomicAdd(p.hist + static_cast<size_t>(t) * kBins + bin_of(__uint_as_float(e.x), smin[r], width[r], inv_width[r]), 1u);
+    const int bin = bin_of(__uint_as_float(e.x), smin[r], width[r], inv_width[r]);
+    if (LT_IN_BOUNDS(bin >= 0 && bin < kBins, p.ctl)) atomicAdd(p.hist + static_cast<size_t>(t) * kBins + bin, 1u);
   }
   __syncwarp();
 }
@@ -216,7 +218,7 @@ knn_scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (!knn_item(p, qb_lo, n_qb, item, it)) continue;
         if (it.qb != cur_qb) {
           // a new query block: wait until the UMMAs of the previous one no longer read it
-          ok = mbar_wait<40>(smem_u32(&st->bar_q_empty), (n_done & 1) ^ 1, abort_flag);
+          ok = mbar_wait<40>(smem_u32(&st->bar_q_empty), (n_done & 1) ^ 1, abort_flag, p.wait_limit_us);
           if (!ok) break;
           mbar_arrive_expect_tx(smem_u32(&st->bar_q_full), n_slices * kQSliceBytes);
           for (int sl = 0; sl < n_slices; ++sl)
@@ -226,7 +228,7 @@ knn_scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
         for (int tile = it.tile_lo; tile < it.tile_hi && ok; ++tile) {
           for (int sl = 0; sl < n_slices; ++sl) {
-            ok = mbar_wait<40>(smem_u32(&st->bar_empty[stage]), phase ^ 1, abort_flag);
+            ok = mbar_wait<40>(smem_u32(&st->bar_empty[stage]), phase ^ 1, abort_flag, p.wait_limit_us);
             if (!ok) break;
             mbar_arrive_expect_tx(smem_u32(&st->bar_full[stage]), kXSliceBytes);
             tma_load_2d(x_base + stage * kXSliceBytes, &tm_x, sl * kSliceElems, tile * kTileKeys, smem_u32(&st->bar_full[stage]));
@@ -250,18 +252,18 @@ knn_scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (!knn_item(p, qb_lo, n_qb, item, it)) continue;
         if (it.qb != cur_qb) {
           if (cur_qb >= 0) tc_commit(smem_u32(&st->bar_q_empty));  // arrives once every UMMA issued so far is done
-          ok = mbar_wait<40>(smem_u32(&st->bar_q_full), n_done & 1, abort_flag);
+          ok = mbar_wait<40>(smem_u32(&st->bar_q_full), n_done & 1, abort_flag, p.wait_limit_us);
           if (!ok) break;
           ++n_done;
           cur_qb = it.qb;
         }
         for (int tile = it.tile_lo; tile < it.tile_hi && ok; ++tile, ++seq) {
           const uint32_t buf = seq & (kAccBufs - 1);
-          ok = mbar_wait<40>(smem_u32(&st->bar_acc_empty[buf]), ((seq >> 2) & 1) ^ 1, abort_flag);
+          ok = mbar_wait<40>(smem_u32(&st->bar_acc_empty[buf]), ((seq >> 2) & 1) ^ 1, abort_flag, p.wait_limit_us);
           if (!ok) break;
           tc_fence_after();
           for (int sl = 0; sl < n_slices; ++sl) {
-            ok = mbar_wait<40>(smem_u32(&st->bar_full[stage]), phase, abort_flag);
+            ok = mbar_wait<40>(smem_u32(&st->bar_full[stage]), phase, abort_flag, p.wait_limit_us);
             if (!ok) break;
             tc_fence_after();
 #pragma unroll
@@ -343,7 +345,11 @@ knn_scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           while (!done) {
             for (int r = 0; r < kQB && !done; ++r) {
               const int t = t0 + r;
-              done = *reinterpret_cast<volatile int*>(&st->done_seq) >= item_seq || *abort_flag;
+              // lane 0 reads the flags and the whole warp follows its decision, so that no lane can leave
+              // while others still execute the full-mask shuffles below
+              int d = 0;
+              if (lane == 0) d = (*reinterpret_cast<volatile int*>(&st->done_seq) >= item_seq || *abort_flag) ? 1 : 0;
+              done = __shfl_sync(0xffffffffu, d, 0) != 0;
               if (done || t < p.row_begin || t >= p.row_end) continue;
               const uint4* hp = reinterpret_cast<const uint4*>(p.hist + static_cast<size_t>(t) * kBins + lane * 8);
               const uint4 h0 = __ldcg(hp), h1 = __ldcg(hp + 1);
@@ -397,7 +403,7 @@ knn_scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           if ((seq & 1u) != set) continue;
           const uint32_t buf = seq & (kAccBufs - 1);
           const int s = tile * kTileKeys + key_in_tile;
-          ok = mbar_wait(smem_u32(&st->bar_acc_full[buf]), (seq >> 2) & 1, abort_flag);
+          ok = mbar_wait(smem_u32(&st->bar_acc_full[buf]), (seq >> 2) & 1, abort_flag, p.wait_limit_us);
           tc_fence_after();
           uint32_t va[32], vb[32];
           tmem_ld32(tlane + buf * kQB, va);
@@ -420,7 +426,8 @@ knn_scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
               // + 0 turns -0 into +0, so that the bit order of the scores is their value order
               const float score = __fadd_rn(__uint_as_float(qq < 32 ? va[qq & 31] : vb[qq & 31]), 0.f);
               const int t = t0 + qq;
-              if (in_range && t >= p.row_begin && t < p.row_end) p.dump[static_cast<size_t>(t - p.row_begin) * p.dump_ld + s] = score;
+              if (in_range && t >= p.row_begin && t < p.row_end && LT_IN_BOUNDS(s >= 0 && s < p.dump_ld, p.ctl))
+                p.dump[static_cast<size_t>(t - p.row_begin) * p.dump_ld + s] = score;
             }
           } else {
             // ---- paper Sec. 3.2 "Filtering": a compare per score (rows outside the launch have thr = +inf;
@@ -519,7 +526,9 @@ cudaError_t knn_launch(const CUtensorMap& tq, const CUtensorMap& tx, const KnnSc
 bool scan_knn_supported(int D) { return D >= kSliceElems && D % kSliceElems == 0 && D <= kKnnMaxSlices * kSliceElems; }
 
 cudaError_t launch_scan_knn(int mode, const void* q, int T, const void* x, long long n_keys_view, long long key_pitch_elems,
-                            const KnnScanParams& p, int grid, cudaStream_t stream) {
+                            const KnnScanParams& params, int grid, cudaStream_t stream) {
+  KnnScanParams p = params;
+  if (p.wait_limit_us == 0) p.wait_limit_us = kDefaultWaitLimitUs;
   CUtensorMap tq, tx;
   if (!knn_map(&tq, q, static_cast<uint64_t>(p.D), static_cast<uint64_t>(T), static_cast<uint64_t>(p.D) * 2, kQB))
     return cudaErrorInvalidValue;

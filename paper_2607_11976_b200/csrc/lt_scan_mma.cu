@@ -126,7 +126,11 @@ __device__ __forceinline__ bool resolve_item(const ScanParams& p, int n_blocks, 
 // Where the scale of view key s lives: at s * ks_stride, or with a paged key cache at the key's physical row.
 template <bool kPaged>
 __device__ __forceinline__ size_t scale_index(const ScanParams& p, int s) {
-  if (kPaged) return static_cast<size_t>(__ldg(p.page_table + (s / kPageKeys))) * kPageKeys + static_cast<size_t>(s % kPageKeys);
+  if (kPaged) {
+    long long phys = __ldg(p.page_table + (s / kPageKeys));
+    if (!LT_IN_BOUNDS(phys >= 0 && phys < p.pool_pages, p.ctl)) phys = 0;  // a page-table entry outside the pool
+    return static_cast<size_t>(phys) * kPageKeys + static_cast<size_t>(s % kPageKeys);
+  }
   return static_cast<size_t>(s) * p.ks_stride;
 }
 
@@ -219,8 +223,10 @@ __device__ __forceinline__ void flush_stage(const uint2* list, int count, const 
   for (int i = lane; i < count; i += 32) {
     const uint2 e = list[i];
     const uint32_t pos = base + i;
-    if (pos < static_cast<uint32_t>(p.cap)) cand[pos] = e;
-    atomicAdd(hist + bin_of(__uint_as_float(e.x), smin, width, inv_width), 1u);
+    if (pos < static_cast<uint32_t>(p.cap) && LT_IN_BOUNDS(t >= 0 && t < p.T && e.y < static_cast<uint32_t>(p.n_keys), p.ctl))
+      cand[pos] = e;
+    const int bin = bin_of(__uint_as_float(e.x), smin, width, inv_width);
+    if (LT_IN_BOUNDS(bin >= 0 && bin < kBins && t >= 0 && t < p.T, p.ctl)) atomicAdd(hist + bin, 1u);
   }
   __syncwarp();
 }
@@ -294,7 +300,7 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         Item it;
         if (!resolve_item(p, n_blocks, item, it)) continue;
         // query block: wait until the UMMAs of the previous item no longer read it
-        ok = mbar_wait<40>(smem_u32(&st->bar_q_empty), (n_done & 1) ^ 1, abort_flag);
+        ok = mbar_wait<40>(smem_u32(&st->bar_q_empty), (n_done & 1) ^ 1, abort_flag, p.wait_limit_us);
         if (!ok) break;
         mbar_arrive_expect_tx(smem_u32(&st->bar_q_full), C::kQBytes);
         for (int u = 0; u < kUnits; ++u)
@@ -303,8 +309,14 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
                         (it.t0 + u * kUnitQ) * kH, smem_u32(&st->bar_q_full));
         ++n_done;
         for (int tile = it.tile_lo; tile < it.tile_hi; ++tile) {
-          ok = mbar_wait<40>(smem_u32(&st->bar_empty[stage]), phase ^ 1, abort_flag);
+          ok = mbar_wait<40>(smem_u32(&st->bar_empty[stage]), phase ^ 1, abort_flag, p.wait_limit_us);
           if (!ok) break;
+          // test hook (lt_tunables.debug_flags): CTA 0 never loads the first key tile of its first item, so
+          // the UMMA warp's wait for it runs out and the whole CTA unwinds through the timeout path
+          if ((p.debug_flags & LT_DEBUG_SKIP_ONE_KTILE) && blockIdx.x == 0 && n_done == 1 && tile == it.tile_lo) {
+            ok = false;
+            break;
+          }
           mbar_arrive_expect_tx(smem_u32(&st->bar_full[stage]), C::kStageBytes);
           if (!kPaged) {
             for (int hf = 0; hf < C::kHalves; ++hf)
@@ -315,7 +327,8 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             // box is then 64 rows); pages past the end of the table are read from page 0 and masked later
             for (int pg = 0; pg < kTileKeys / kPageKeys; ++pg) {
               const int lp = tile * (kTileKeys / kPageKeys) + pg;
-              const int phys = lp < p.n_pages ? __ldg(p.page_table + lp) : 0;
+              int phys = lp < p.n_pages ? __ldg(p.page_table + lp) : 0;
+              if (!LT_IN_BOUNDS(phys >= 0 && phys < p.pool_pages, p.ctl)) phys = 0;  // entry outside the pool
               for (int hf = 0; hf < C::kHalves; ++hf)
                 tma_load_2d(k_base + stage * C::kStageBytes + hf * kSwizzleTile + pg * kPageKeys * 128, &tm_k,
                             hf * C::kElemsPerRow128, phys * kPageKeys, smem_u32(&st->bar_full[stage]));
@@ -340,14 +353,14 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
         Item it;
         if (!resolve_item(p, n_blocks, item, it)) continue;
-        ok = mbar_wait<40>(smem_u32(&st->bar_q_full), n_done & 1, abort_flag);
+        ok = mbar_wait<40>(smem_u32(&st->bar_q_full), n_done & 1, abort_flag, p.wait_limit_us);
         if (!ok) break;
         ++n_done;
         for (int tile = it.tile_lo; tile < it.tile_hi && ok; ++tile) {
-          ok = mbar_wait<40>(smem_u32(&st->bar_full[stage]), phase, abort_flag);
+          ok = mbar_wait<40>(smem_u32(&st->bar_full[stage]), phase, abort_flag, p.wait_limit_us);
           if (!ok) break;
           for (int u = 0; u < kUnits; ++u) {
-            ok = mbar_wait<40>(smem_u32(&st->bar_tmem_empty[u]), acc_phase ^ 1, abort_flag);
+            ok = mbar_wait<40>(smem_u32(&st->bar_tmem_empty[u]), acc_phase ^ 1, abort_flag, p.wait_limit_us);
             if (!ok) break;
             tc_fence_after();
 #pragma unroll
@@ -467,11 +480,15 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
                 }
               }
             }
-            // sleep in slices so that the end of the item is noticed quickly
+            // sleep in slices so that the end of the item is noticed quickly; lane 0 reads the flags and the
+            // whole warp follows its decision, so that no lane can leave while others still execute the
+            // full-mask shuffles above
             bool done = false;
             for (unsigned int slept = 0; slept < sleep_ns && !done; slept += 1000) {
               __nanosleep(1000);
-              done = *reinterpret_cast<volatile int*>(&st->done_seq) >= seq || *abort_flag;
+              int d = 0;
+              if (lane == 0) d = (*reinterpret_cast<volatile int*>(&st->done_seq) >= seq || *abort_flag) ? 1 : 0;
+              done = __shfl_sync(0xffffffffu, d, 0) != 0;
             }
             if (done) break;
             if (sleep_ns < 32000) sleep_ns += sleep_ns >> 1;
@@ -506,7 +523,7 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             const int r = u * kUnitQ + g;
             float thr = 0.f;
             if (kMode == kModeFilter) thr = *reinterpret_cast<volatile float*>(&st->thr[r]);
-            ok = mbar_wait(smem_u32(&st->bar_tmem_full[u]), acc_phase, abort_flag);
+            ok = mbar_wait(smem_u32(&st->bar_tmem_full[u]), acc_phase, abort_flag, p.wait_limit_us);
             tc_fence_after();
             // the 64 columns of this query: both loads in flight, one wait.  The loads are issued even
             // after a failed wait (they then fetch values nobody uses): keeping them unconditional
@@ -530,7 +547,8 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             const float score = combine(acc, ks);
             if (kMode == kModeDump) {
               const int dr = st->dump_row[r];
-              if (dr >= 0 && s < p.n_keys)
+              if (dr >= 0 && s < p.n_keys &&
+                  LT_IN_BOUNDS(s < p.dump_ld && dr < (p.fb_list != nullptr ? p.fb_slots * kBlockQ : p.row_end - p.row_begin), p.ctl))
                 p.dump[static_cast<size_t>(dr) * p.dump_ld + s] = (s < st->vis[r]) ? score : -INFINITY;
             } else {
               // ---- paper Sec. 3.2 "Filtering": gate, ballot-compact into the warp's staging list,
@@ -636,12 +654,40 @@ cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const ScanParam
 
 }  // namespace
 
+namespace {
+__global__ void wait_timeout_probe_kernel(unsigned int limit_us, int* result2) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    fence_mbar_init();
+  }
+  __syncthreads();
+  // phase 0 of `bar` never completes: the wait can only end by its time limit
+  const bool ok = mbar_wait<40>(smem_u32(&bar), 0, &abort_flag, limit_us);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    result2[0] = ok ? 1 : 0;
+    result2[1] = abort_flag;
+  }
+}
+}  // namespace
+
+cudaError_t launch_wait_timeout_probe(unsigned int limit_us, int* result2, cudaStream_t stream) {
+  wait_timeout_probe_kernel<<<1, 32, 0, stream>>>(limit_us, result2);
+  return cudaGetLastError();
+}
+
 bool scan_mma_supported(int dtype, int H, int D) {
   return (dtype == LT_DTYPE_BF16 || dtype == LT_DTYPE_E4M3) && H == kH && D == kD;
 }
 
 cudaError_t launch_scan_mma(int dtype, int mode, const void* q, int T, const void* k, long long n_keys_view,
-                            long long key_pitch_elems, const ScanParams& p, int grid, cudaStream_t stream) {
+                            long long key_pitch_elems, const ScanParams& params, int grid, cudaStream_t stream) {
+  ScanParams p = params;
+  if (p.wait_limit_us == 0) p.wait_limit_us = kDefaultWaitLimitUs;
+  if (mode != kModeFilter) p.debug_flags = 0;  // the test hooks act on the fused scan only
   const bool fp8 = (dtype == LT_DTYPE_E4M3);
   const size_t esz = fp8 ? 1 : 2;
   CUtensorMap tq, tk;

@@ -257,7 +257,7 @@ __device__ __forceinline__ uint64_t* radix_sort_by_score_desc(uint64_t* src, uin
 // by the radix passes above, and by the bitonic network only if equal scores were left in the wrong order.
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ void sort_and_write(uint64_t* sel, int count, int topk, int32_t* out_idx, float* out_score,
-                                               uint64_t* alt = nullptr) {
+                                               int n_keys, Control* ctl, uint64_t* alt = nullptr) {
   bool sorted = false;
   if (alt != nullptr && count >= 512 && count <= kRadixSortMax) sel = radix_sort_by_score_desc(sel, alt, count, &sorted);
   if (!sorted) {
@@ -268,6 +268,7 @@ __device__ __forceinline__ void sort_and_write(uint64_t* sel, int count, int top
   }
   for (int j = threadIdx.x; j < topk; j += blockDim.x) {
     bool have = j < count;
+    if (have && !LT_IN_BOUNDS(key_index(sel[j]) >= 0 && key_index(sel[j]) < n_keys, ctl)) have = false;  // never publish an index outside the keys
     out_idx[j] = have ? key_index(sel[j]) : -1;
     if (out_score != nullptr) out_score[j] = have ? key_score(sel[j]) : -INFINITY;
   }
@@ -554,7 +555,8 @@ __global__ void __launch_bounds__(kFinalThreads) final_select_kernel(const Final
         keys = radix_sort_by_score_desc(sel, alt, n_keep, &sorted);
         if (sorted) {
           for (int j = threadIdx.x; j < p.topk; j += kFinalThreads) {
-            const bool have = j < kk;
+            bool have = j < kk;
+            if (have && !LT_IN_BOUNDS(key_index(keys[j]) >= 0 && key_index(keys[j]) < p.N, p.ctl)) have = false;
             out_idx[j] = have ? key_index(keys[j]) : -1;
             if (out_score != nullptr) out_score[j] = have ? key_score(keys[j]) : -INFINITY;
           }
@@ -568,7 +570,7 @@ __global__ void __launch_bounds__(kFinalThreads) final_select_kernel(const Final
         keep_top_keys(keys, n_keep, kk, hist, &s_count);
         n_keep = kk;
       }
-      sort_and_write(keys, n_keep, p.topk, out_idx, out_score, keys == sel ? alt : nullptr);
+      sort_and_write(keys, n_keep, p.topk, out_idx, out_score, p.N, p.ctl, keys == sel ? alt : nullptr);
       return;
     }
   }
@@ -613,7 +615,7 @@ __global__ void __launch_bounds__(kSelThreads) select_rows_kernel(const SelectRo
     // every visible key is selected
     for (int i = tid; i < vis; i += kSelThreads) sel[i] = pack_key(row[i], i);
     __syncthreads();
-    sort_and_write(sel, vis, p.topk, out_idx, out_score);
+    sort_and_write(sel, vis, p.topk, out_idx, out_score, p.N, p.ctl);
     return;
   }
 
@@ -739,7 +741,7 @@ __global__ void __launch_bounds__(kSelThreads) select_rows_kernel(const SelectRo
    }
   }
   __syncthreads();
-  sort_and_write(sel, kk, p.topk, out_idx, out_score);
+  sort_and_write(sel, kk, p.topk, out_idx, out_score, p.N, p.ctl);
 }
 
 }  // namespace
