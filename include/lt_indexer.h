@@ -322,6 +322,9 @@ int lt_indexer_topk_static(int dtype, const void* q, const float* w, const void*
                            int T, int N, int H, int D, int topk, int causal_offset,
                            int32_t* out_idx, float* out_score, void* stream);
 
+/* Largest N lt_indexer_topk_static accepts: (LT_STATIC_SCRATCH_BYTES - 256) / 4 keys (no counterpart in the paper). */
+int lt_indexer_topk_static_max_keys(void);
+
 /*
  * Copies the 8-int status block of a workspace to host memory after synchronising
  * `stream`: [0] LT_STATUS_* bits, [1] rows that took the fallback, [2] largest

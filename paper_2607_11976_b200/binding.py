@@ -103,6 +103,7 @@ def load() -> ctypes.CDLL:
     lib.lt_indexer_topk_static.restype = i
     lib.lt_read_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int), vp]
     lib.lt_read_status.restype = i
+    lib.lt_indexer_topk_static_max_keys.restype = i
     lib.lt_read_status_static.argtypes = [ctypes.POINTER(ctypes.c_int), vp]
     lib.lt_read_status_static.restype = i
     lib.lt_debug_wait_timeout.argtypes = [i, ip, vp]

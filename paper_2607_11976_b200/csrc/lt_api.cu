@@ -948,6 +948,8 @@ int lt_read_status(const void* workspace, int* status8_host, void* stream) {
   return LT_OK;
 }
 
+int lt_indexer_topk_static_max_keys(void) { return static_cast<int>((kStaticScratchBytes - kAlign) / 4); }
+
 int lt_read_status_static(int* status8_host, void* stream) {
   if (status8_host == nullptr) return LT_ERR_INVALID_ARG;
   void* base = nullptr;

@@ -42,6 +42,27 @@ def test_static_entry_matches_regular_entry_twice_in_a_row():
         assert np.array_equal(got_score.view(np.uint32), want_score.view(np.uint32))
 
 
+def test_static_entry_runs_several_passes_over_its_fixed_array():
+    """A row of 600,000 scores takes 2.4 MB of the 16 MiB array: 6 rows per pass, four passes, the later
+    ones starting at rows that are no multiple of the scan's 8-row blocks.  Same bits as the regular entry,
+    a clean status block, and no device memory taken or returned by the call."""
+    inp = make_config("dsa_bf16", T=20, N=600000, topk=64)
+    want_idx, want_score, _ = run_topk(inp)
+    q, w, k, ks = lt.to_device(inp)
+    out_idx = torch.full((inp.T, inp.topk), -7, dtype=torch.int32, device="cuda")
+    out_score = torch.full((inp.T, inp.topk), float("nan"), dtype=torch.float32, device="cuda")
+    lt.lt_indexer_topk_static(inp.dtype, q, w, k, ks, inp.topk, inp.causal_offset, out_idx, out_score)  # loads the kernels
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    lt.lt_indexer_topk_static(inp.dtype, q, w, k, ks, inp.topk, inp.causal_offset, out_idx, out_score)
+    status = lt.lt_read_status_static()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, "the allocation-free entry point changed the device's free memory"
+    assert status[0] & (lt.LT_STATUS_TIMEOUT | lt.LT_STATUS_BOUNDS) == 0
+    assert np.array_equal(out_idx.cpu().numpy(), want_idx)
+    assert np.array_equal(out_score.cpu().numpy().view(np.uint32), want_score.view(np.uint32))
+
+
 def test_static_entry_rejects_what_does_not_fit():
     lib = lt.load()
     fake = ctypes.c_void_p(0x1000)
@@ -49,4 +70,8 @@ def test_static_entry_rejects_what_does_not_fit():
     n_too_big = (16 << 20) // 4  # one row of N floats no longer fits behind the 256-byte status block
     rc = lib.lt_indexer_topk_static(1, fake, fake, fake, null, 8, n_too_big, 64, 128, 4, n_too_big - 8, fake, null, null)
     assert rc == -5 and b"fixed scratch" in lib.lt_strerror(rc)
+    n_max = lib.lt_indexer_topk_static_max_keys()
+    assert n_max == ((16 << 20) - 256) // 4 == 4194240
+    # one key more than the largest accepted N is refused before anything is enqueued
+    assert lib.lt_indexer_topk_static(1, fake, fake, fake, null, 8, n_max + 1, 64, 128, 4, n_max - 7, fake, null, null) == -5
     assert lib.lt_indexer_topk_static(1, null, fake, fake, null, 8, 64, 64, 128, 4, 56, fake, null, null) == -1
