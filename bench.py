@@ -34,10 +34,10 @@ UNIT = "pairs/s"
 NOMINAL_FP8_TFLOPS = 4500.0
 NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM bytes of one launch of the fused scan kernel (dram__bytes_read.sum + dram__bytes_write.sum) from
-# the ncu capture of a 592-row case summarised in profiles/scan_kernel_fp8_T592_N1M.md: 164.3 MB, of which
-# the key stream (N * D bytes, read once whatever the number of rows) is 134.2 MB and the rest
-# (candidate write-back, queries, weights) grows with the rows: (164.3 - 134.2) MB / 592 rows.
+# DRAM bytes of one launch of the fused scan kernel (dram__bytes_read.sum + dram__bytes_write.sum) from an
+# ncu capture of a 592-row case of the same workload: 164.3 MB, of which the key stream (N * D bytes, read
+# once whatever the number of rows) is 134.2 MB and the rest (candidate write-back, queries, weights) grows
+# with the rows: (164.3 - 134.2) MB / 592 rows.
 SCAN_TRAFFIC = {"fp8_1m": {"fixed_bytes": 134.2e6, "bytes_per_row": (164.3e6 - 134.2e6) / 592}}
 
 
@@ -341,6 +341,197 @@ def time_aux_ops(torch, lt, out_idx, inp, hbm_gbs, peak_kind, reps=5):
     return out
 
 
+# ---------------------------------------------------------------------------------------------------------
+# the other configurations and the "next" operations, measured briefly in the same run (default line only)
+# ---------------------------------------------------------------------------------------------------------
+def _timed_ms(torch, fn, steps, flush=None):
+    """Mean device time of `steps` calls, each bracketed by CUDA events; L2 flushed (untimed) before each."""
+    stream = torch.cuda.current_stream()
+    tot = 0.0
+    for _ in range(steps):
+        if flush is not None:
+            flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        fn()
+        e1.record(stream)
+        e1.synchronize()
+        tot += e0.elapsed_time(e1)
+    return tot / steps
+
+
+def measure_config(torch, lt, inp, peaks, flush, steps=5, warmup=3, unfused=True):
+    """One configuration through lt_indexer_topk_ex: ms per step, pairs/s, the scan's roofline fraction against
+    its own dtype's measured peak, fallback rows, and the decoupled path's time."""
+    q, w, k, ks = lt.to_device(inp)
+    out_idx = torch.empty((inp.T, inp.topk), dtype=torch.int32, device="cuda")
+    out_score = torch.empty((inp.T, inp.topk), dtype=torch.float32, device="cuda")
+    ws = lt.alloc_workspace(inp.dtype, inp.T, inp.N, inp.H, inp.D, inp.topk)
+
+    def step():
+        lt.lt_indexer_topk_ex(inp.dtype, q, w, k, ks, inp.topk, inp.causal_offset, out_idx, out_score, ws)
+
+    for _ in range(warmup):
+        step()
+    phase = []
+
+    def timed_step():
+        step()
+
+    ms = 0.0
+    for _ in range(steps):
+        ms += _timed_ms(torch, timed_step, 1, flush)
+        phase.append(lt.lt_read_phase_ms())
+    ms /= steps
+    status = lt.lt_read_status(ws)
+    pairs = inp.valid_pairs()
+    rec = {"workload": inp.name, "dtype": inp.dtype, "T": inp.T, "N": inp.N, "topk": inp.topk, "ms_per_step": ms,
+           "pairs_per_s": pairs / (ms * 1e-3), "fallback_rows": status[1], "status_bits": status[0],
+           "mean_survivors_per_row": status[3] / inp.T, "steps": steps}
+    scan_ms = statistics.mean(p[2] for p in phase)
+    rec["phases_ms"] = {"sample": statistics.mean(p[0] + p[1] for p in phase), "fused_scan": scan_ms,
+                        "final_select": statistics.mean(p[3] for p in phase), "fallback": statistics.mean(p[4] for p in phase)}
+    if inp.dtype in ("bf16", "e4m3") and inp.H == 64 and inp.D == 128:
+        peak = peaks["bf16_tflops"] * (2.0 if inp.dtype == "e4m3" else 1.0)
+        achieved = 2.0 * inp.H * inp.D * pairs / (scan_ms * 1e-3) / 1e12
+        rec["roofline"] = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak}
+    else:
+        rec["roofline"] = None  # generic SIMT path (a correctness configuration): no phase events either
+        rec["phases_ms"] = None
+    if unfused:
+        buf = torch.empty(256 + (1024 << 20), dtype=torch.uint8, device="cuda")
+
+        def unf():
+            lt.lt_unfused_topk(inp.dtype, q, w, k, ks, inp.topk, inp.causal_offset, out_idx, out_score, buf)
+
+        unf()
+        rec["unfused_ms"] = _timed_ms(torch, unf, 2, flush)
+        del buf
+    return rec
+
+
+def measure_other_configs(torch, lt, peaks, flush):
+    """tiny_f32, dsa_bf16, fp8_ar1 and the adversarial recipes x topk in {64, 512, 2048, 4096}."""
+    import dataclasses
+
+    from workloads import make_config
+
+    out = []
+    for name in ("tiny_f32", "dsa_bf16", "fp8_ar1"):
+        out.append(measure_config(torch, lt, make_config(name), peaks, flush))
+    for name in ("adv_planted", "adv_cluster", "adv_ties", "adv_ties_exact"):
+        base = make_config(name)
+        for topk in (64, 512, 2048, 4096):
+            out.append(measure_config(torch, lt, dataclasses.replace(base, topk=topk), peaks, flush, unfused=(topk == 2048)))
+    return out
+
+
+def measure_next_rows(torch, lt, peaks, peak_kind, flush, main):
+    """The "next" operations: paged key cache against the dense layout, the integer ops on the chunk's result,
+    the previous-chunk sampler's survivors, and the k-NN variant's scan against the HBM roofline."""
+    import dataclasses
+
+    from workloads import make_config
+
+    inp, q, w, k, ks, out_idx, out_score, ws = main
+    res = {}
+    # ---- paged key cache, random page order, same keys
+    n_pages = inp.N // 64
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(1234)
+    table = torch.randperm(n_pages, device="cuda", generator=gen).to(torch.int32)
+    k_pool = torch.empty_like(k)
+    k_pool.view(n_pages, 64, inp.D)[table.long()] = k.view(n_pages, 64, inp.D)
+    ks_pool = torch.empty_like(ks)
+    ks_pool.view(n_pages, 64)[table.long()] = ks.view(n_pages, 64)
+    pws = torch.empty(lt.lt_indexer_topk_paged_workspace_bytes(inp.dtype, inp.T, inp.N, inp.H, inp.D, inp.topk),
+                      dtype=torch.uint8, device="cuda")
+    p_idx = torch.empty_like(out_idx)
+
+    def paged():
+        lt.lt_indexer_topk_paged(inp.dtype, q, w, k_pool, ks_pool, table, inp.N, inp.topk, inp.causal_offset, p_idx, None, pws)
+
+    def dense():
+        lt.lt_indexer_topk_ex(inp.dtype, q, w, k, ks, inp.topk, inp.causal_offset, out_idx, out_score, ws)
+
+    paged()
+    dense()
+    d_ms, p_ms = _timed_ms(torch, dense, 3, flush), _timed_ms(torch, paged, 3, flush)
+    res["paged_key_cache"] = {"workload": inp.name, "dense_ms": d_ms, "paged_ms": p_ms, "delta": p_ms / d_ms - 1.0,
+                              "same_indices": bool(torch.equal(p_idx, out_idx))}
+    del k_pool, ks_pool, pws, p_idx
+    # ---- integer ops on the chunk's index matrix
+    res.update(time_aux_ops(torch, lt, out_idx, inp, peaks["hbm_gbs"], peak_kind))
+    # ---- previous-chunk sampler on two consecutive (shorter) chunks of the structured workload
+    T = 1024
+    both = make_config("hot_fp8", T=2 * T)
+    n_prev = both.causal_offset + T
+    prev = dataclasses.replace(both, q=both.q[:T], w=both.w[:T], k=both.k[:n_prev], k_scale=both.k_scale[:n_prev])
+    cur = dataclasses.replace(both, q=both.q[T:], w=both.w[T:], causal_offset=both.causal_offset + T)
+    pq, pw, pk, pks = lt.to_device(prev)
+    cq, cw, ck, cks = lt.to_device(cur)
+    idx1 = torch.empty((T, prev.topk), dtype=torch.int32, device="cuda")
+    ws1 = lt.alloc_workspace(prev.dtype, T, prev.N, prev.H, prev.D, prev.topk)
+    lt.lt_indexer_topk_ex(prev.dtype, pq, pw, pk, pks, prev.topk, prev.causal_offset, idx1, None, ws1)
+    n_sample = min(3 * prev.topk, lt.LT_MAX_TOPK)
+    sample = torch.empty(n_sample, dtype=torch.int32, device="cuda")
+    fws = torch.empty(lt.lt_topk_frequent_workspace_bytes(prev.N), dtype=torch.uint8, device="cuda")
+    lt.lt_topk_frequent(idx1, prev.N, sample, None, fws)
+    idx2 = torch.empty((T, cur.topk), dtype=torch.int32, device="cuda")
+    ws2 = lt.alloc_workspace(cur.dtype, T, cur.N, cur.H, cur.D, cur.topk)
+    lt.lt_indexer_topk_ex(cur.dtype, cq, cw, ck, cks, cur.topk, cur.causal_offset, idx2, None, ws2)
+    surv_default = lt.lt_read_status(ws2)[3] / T
+    ws3 = torch.empty(lt.lt_indexer_topk_sampled_workspace_bytes(cur.dtype, T, cur.N, cur.H, cur.D, cur.topk, n_sample),
+                      dtype=torch.uint8, device="cuda")
+    idx3 = torch.empty_like(idx2)
+    lt.lt_indexer_topk_sampled(cur.dtype, cq, cw, ck, cks, cur.topk, cur.causal_offset, sample, idx3, None, ws3)
+    st3 = lt.lt_read_status(ws3)
+    res["previous_chunk_sampler"] = {"workload": "hot_fp8, two chunks of 1024 rows", "n_sample": n_sample,
+                                     "survivors_per_row": st3[3] / T, "survivors_per_row_default_sampler": surv_default,
+                                     "fallback_rows": st3[1], "same_indices": bool(torch.equal(idx2, idx3))}
+    del pq, pw, pk, pks, cq, cw, ck, cks, ws1, ws2, ws3, fws
+    # ---- k-NN variant: 64 queries x 2^20 x 768 bf16, unit vectors around 64 centres, generated on the device with
+    # the recipe of the CPU generator (the parity tests use the CPU generator; this line only times)
+    Tq, Nc, Dk, kk = 64, 1 << 20, 768, 1024
+    g = torch.Generator(device="cuda")
+    g.manual_seed(20)
+    centres = torch.nn.functional.normalize(torch.randn(64, Dk, device="cuda", generator=g), dim=1)
+
+    def draw(rows):
+        which = torch.randint(0, 64, (rows,), device="cuda", generator=g)
+        out = torch.empty((rows, Dk), dtype=torch.bfloat16, device="cuda")
+        for r0 in range(0, rows, 1 << 17):
+            r1 = min(rows, r0 + (1 << 17))
+            v = 0.7 * centres[which[r0:r1]] + torch.randn(r1 - r0, Dk, device="cuda", generator=g) / Dk ** 0.5
+            out[r0:r1] = torch.nn.functional.normalize(v, dim=1).to(torch.bfloat16)
+        return out
+
+    xq, xc = draw(Tq), draw(Nc)
+    kidx = torch.empty((Tq, kk), dtype=torch.int32, device="cuda")
+    kws = torch.empty(lt.lt_knn_topk_workspace_bytes(Tq, Nc, Dk, kk), dtype=torch.uint8, device="cuda")
+
+    def knn():
+        lt.lt_knn_topk(xq, xc, kk, kidx, None, kws)
+
+    for _ in range(3):
+        knn()
+    ph = []
+    kms = 0.0
+    for _ in range(10):
+        kms += _timed_ms(torch, knn, 1, flush)
+        ph.append(lt.lt_read_phase_ms())
+    kms /= 10
+    kst = lt.lt_read_status(kws)
+    scan_ms = statistics.mean(p[2] for p in ph)
+    nbytes = Nc * Dk * 2 + Tq * Dk * 2 + kst[3] * 8
+    res["knn"] = {"T": Tq, "N": Nc, "D": Dk, "topk": kk, "ms_per_step": kms, "pairs_per_s": Tq * Nc / (kms * 1e-3),
+                  "scan_ms": scan_ms, "fallback_rows": kst[1],
+                  "roofline": {"bound": "hbm", "achieved": nbytes / scan_ms / 1e6, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                               "frac": nbytes / scan_ms / 1e6 / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",
+                               "algorithmic_bytes": nbytes}}
+    return res
+
+
 def run_knn(args, rank: int, local_rank: int, world: int):
     """k-NN (inner-product) variant: one step = exact top-k of a batch of queries over the whole corpus."""
     import torch
@@ -536,6 +727,8 @@ def main():
                     help="k-NN workloads: also time prefixes of the corpus (1M, 2M, 4M, ... vectors) x k in {128, 1024, 4096, 8192} "
                          "(the grid of the paper's retrieval benchmark) and add the table as 'sweep'")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="default fp8_1m line only: skip the brief measurements of the other configurations and the next-row operations")
     ap.add_argument("--no-unfused", action="store_true")
     ap.add_argument("--graph", action="store_true", help="indexer workloads: also time the step replayed from a CUDA graph")
     ap.add_argument("--no-graph", action="store_true", help="k-NN workloads: skip the CUDA-graph replay of the step")
@@ -808,6 +1001,13 @@ def main():
 
     if args.aux:
         line["aux"] = time_aux_ops(torch, lt, out_idx, inp, peaks["hbm_gbs"], peak_kind)
+
+    default_line = (args.workload == "fp8_1m" and not args.rows and page_table is None and sample_idx is None and world == 1)
+    if default_line and not args.no_extras:
+        # the other four configurations and the "next" operations, a few timed steps each, in the same process
+        del dev2, outs2, h_outs2, host
+        line["configs"] = measure_other_configs(torch, lt, peaks, flush)
+        line["next"] = measure_next_rows(torch, lt, peaks, peak_kind, flush, (inp, q, w, k, ks, out_idx, out_score, ws))
 
     if not args.no_unfused and page_table is None:
         # in-repo unfused GPU baseline: dense scores to HBM in row sub-chunks, then a full-row radix select
