@@ -41,11 +41,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait: gives up after `limit_us` microseconds of wall time or as soon as *abort_flag is set by
-// anyone.  Returns false on give-up (and sets *abort_flag), so callers can unwind without hanging the GPU.
+// Bounded wait: gives up after abort_flag[1] microseconds of wall time or as soon as abort_flag[0] is set by
+// anyone.  Returns false on give-up (and sets abort_flag[0]), so callers can unwind without hanging the GPU.
+// The limit sits next to the flag, in shared memory, so that only the slow path ever reads it.
 constexpr uint32_t kDefaultWaitLimitUs = 2000000u;  // 2 s
 template <int kBackoffNs = 0>
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t limit_us) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   uint64_t t0 = 0;
   for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -55,7 +56,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       uint64_t now = globaltimer_ns();
       if (t0 == 0) {
         t0 = now;
-      } else if (now - t0 > static_cast<uint64_t>(limit_us) * 1000ull) {
+      } else if (now - t0 > static_cast<uint64_t>(static_cast<uint32_t>(abort_flag[1])) * 1000ull) {
         *abort_flag = 1;
         return false;
       }

@@ -58,7 +58,8 @@ struct KnnTail {
   uint64_t bar_acc_full[kAccBufs];
   uint64_t bar_acc_empty[kAccBufs];
   uint32_t tmem_base;
-  int abort_flag;
+  int abort_flag;     // [0] raised by a wait that ran out; every role unwinds on it
+  int wait_limit_us;  // [1] bound of every wait (read by mbar_wait through the flag's address)
   int epi_abort;
   int done_seq;
   uint4 stage[kKnnEpiWarps][kKnnStageLen];  // per warp: (score bits, corpus index, query row, -) of survivors
@@ -185,6 +186,7 @@ knn_scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       mbar_init(smem_u32(&st->bar_acc_empty[i]), 4);  // the four quarter warps of the set that drains the tile
     }
     st->abort_flag = 0;
+    st->wait_limit_us = static_cast<int>(p.wait_limit_us);
     st->epi_abort = 0;
     st->done_seq = 0;
     fence_mbar_init();
@@ -218,7 +220,7 @@ knn_scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (!knn_item(p, qb_lo, n_qb, item, it)) continue;
         if (it.qb != cur_qb) {
           // a new query block: wait until the UMMAs of the previous one no longer read it
-          ok = mbar_wait<40>(smem_u32(&st->bar_q_empty), (n_done & 1) ^ 1, abort_flag, p.wait_limit_us);
+          ok = mbar_wait<40>(smem_u32(&st->bar_q_empty), (n_done & 1) ^ 1, abort_flag);
           if (!ok) break;
           mbar_arrive_expect_tx(smem_u32(&st->bar_q_full), n_slices * kQSliceBytes);
           for (int sl = 0; sl < n_slices; ++sl)
@@ -228,7 +230,7 @@ knn_scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
         for (int tile = it.tile_lo; tile < it.tile_hi && ok; ++tile) {
           for (int sl = 0; sl < n_slices; ++sl) {
-            ok = mbar_wait<40>(smem_u32(&st->bar_empty[stage]), phase ^ 1, abort_flag, p.wait_limit_us);
+            ok = mbar_wait<40>(smem_u32(&st->bar_empty[stage]), phase ^ 1, abort_flag);
             if (!ok) break;
             mbar_arrive_expect_tx(smem_u32(&st->bar_full[stage]), kXSliceBytes);
             tma_load_2d(x_base + stage * kXSliceBytes, &tm_x, sl * kSliceElems, tile * kTileKeys, smem_u32(&st->bar_full[stage]));
@@ -252,18 +254,18 @@ knn_scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (!knn_item(p, qb_lo, n_qb, item, it)) continue;
         if (it.qb != cur_qb) {
           if (cur_qb >= 0) tc_commit(smem_u32(&st->bar_q_empty));  // arrives once every UMMA issued so far is done
-          ok = mbar_wait<40>(smem_u32(&st->bar_q_full), n_done & 1, abort_flag, p.wait_limit_us);
+          ok = mbar_wait<40>(smem_u32(&st->bar_q_full), n_done & 1, abort_flag);
           if (!ok) break;
           ++n_done;
           cur_qb = it.qb;
         }
         for (int tile = it.tile_lo; tile < it.tile_hi && ok; ++tile, ++seq) {
           const uint32_t buf = seq & (kAccBufs - 1);
-          ok = mbar_wait<40>(smem_u32(&st->bar_acc_empty[buf]), ((seq >> 2) & 1) ^ 1, abort_flag, p.wait_limit_us);
+          ok = mbar_wait<40>(smem_u32(&st->bar_acc_empty[buf]), ((seq >> 2) & 1) ^ 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
           for (int sl = 0; sl < n_slices; ++sl) {
-            ok = mbar_wait<40>(smem_u32(&st->bar_full[stage]), phase, abort_flag, p.wait_limit_us);
+            ok = mbar_wait<40>(smem_u32(&st->bar_full[stage]), phase, abort_flag);
             if (!ok) break;
             tc_fence_after();
 #pragma unroll
@@ -403,7 +405,7 @@ knn_scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           if ((seq & 1u) != set) continue;
           const uint32_t buf = seq & (kAccBufs - 1);
           const int s = tile * kTileKeys + key_in_tile;
-          ok = mbar_wait(smem_u32(&st->bar_acc_full[buf]), (seq >> 2) & 1, abort_flag, p.wait_limit_us);
+          ok = mbar_wait(smem_u32(&st->bar_acc_full[buf]), (seq >> 2) & 1, abort_flag);
           tc_fence_after();
           uint32_t va[32], vb[32];
           tmem_ld32(tlane + buf * kQB, va);

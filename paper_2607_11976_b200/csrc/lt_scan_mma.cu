@@ -80,7 +80,8 @@ struct SmemTail {
   uint64_t bar_tmem_full[2];
   uint64_t bar_tmem_empty[2];
   uint32_t tmem_base;
-  int abort_flag;
+  int abort_flag;     // [0] raised by a wait that ran out; every role unwinds on it
+  int wait_limit_us;  // [1] bound of every wait (read by mbar_wait through the flag's address)
   int epi_abort;
   int done_seq;
   uint2 stage[kEpiWarps][kUnits][kStageLen];  // per warp and unit: (score bits, key index) of survivors
@@ -261,6 +262,7 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       mbar_init(smem_u32(&st->bar_tmem_empty[i]), kEpiWarps);
     }
     st->abort_flag = 0;
+    st->wait_limit_us = static_cast<int>(p.wait_limit_us);
     st->epi_abort = 0;
     st->done_seq = 0;
     fence_mbar_init();
@@ -300,7 +302,7 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         Item it;
         if (!resolve_item(p, n_blocks, item, it)) continue;
         // query block: wait until the UMMAs of the previous item no longer read it
-        ok = mbar_wait<40>(smem_u32(&st->bar_q_empty), (n_done & 1) ^ 1, abort_flag, p.wait_limit_us);
+        ok = mbar_wait<40>(smem_u32(&st->bar_q_empty), (n_done & 1) ^ 1, abort_flag);
         if (!ok) break;
         mbar_arrive_expect_tx(smem_u32(&st->bar_q_full), C::kQBytes);
         for (int u = 0; u < kUnits; ++u)
@@ -309,7 +311,7 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
                         (it.t0 + u * kUnitQ) * kH, smem_u32(&st->bar_q_full));
         ++n_done;
         for (int tile = it.tile_lo; tile < it.tile_hi; ++tile) {
-          ok = mbar_wait<40>(smem_u32(&st->bar_empty[stage]), phase ^ 1, abort_flag, p.wait_limit_us);
+          ok = mbar_wait<40>(smem_u32(&st->bar_empty[stage]), phase ^ 1, abort_flag);
           if (!ok) break;
           // test hook (lt_tunables.debug_flags): CTA 0 never loads the first key tile of its first item, so
           // the UMMA warp's wait for it runs out and the whole CTA unwinds through the timeout path
@@ -353,14 +355,14 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
         Item it;
         if (!resolve_item(p, n_blocks, item, it)) continue;
-        ok = mbar_wait<40>(smem_u32(&st->bar_q_full), n_done & 1, abort_flag, p.wait_limit_us);
+        ok = mbar_wait<40>(smem_u32(&st->bar_q_full), n_done & 1, abort_flag);
         if (!ok) break;
         ++n_done;
         for (int tile = it.tile_lo; tile < it.tile_hi && ok; ++tile) {
-          ok = mbar_wait<40>(smem_u32(&st->bar_full[stage]), phase, abort_flag, p.wait_limit_us);
+          ok = mbar_wait<40>(smem_u32(&st->bar_full[stage]), phase, abort_flag);
           if (!ok) break;
           for (int u = 0; u < kUnits; ++u) {
-            ok = mbar_wait<40>(smem_u32(&st->bar_tmem_empty[u]), acc_phase ^ 1, abort_flag, p.wait_limit_us);
+            ok = mbar_wait<40>(smem_u32(&st->bar_tmem_empty[u]), acc_phase ^ 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
 #pragma unroll
@@ -523,7 +525,7 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             const int r = u * kUnitQ + g;
             float thr = 0.f;
             if (kMode == kModeFilter) thr = *reinterpret_cast<volatile float*>(&st->thr[r]);
-            ok = mbar_wait(smem_u32(&st->bar_tmem_full[u]), acc_phase, abort_flag, p.wait_limit_us);
+            ok = mbar_wait(smem_u32(&st->bar_tmem_full[u]), acc_phase, abort_flag);
             tc_fence_after();
             // the 64 columns of this query: both loads in flight, one wait.  The loads are issued even
             // after a failed wait (they then fetch values nobody uses): keeping them unconditional
@@ -657,19 +659,20 @@ cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const ScanParam
 namespace {
 __global__ void wait_timeout_probe_kernel(unsigned int limit_us, int* result2) {
   __shared__ uint64_t bar;
-  __shared__ int abort_flag;
+  __shared__ int abort_flag[2];  // flag, limit in microseconds
   if (threadIdx.x == 0) {
     mbar_init(smem_u32(&bar), 1);
-    abort_flag = 0;
+    abort_flag[0] = 0;
+    abort_flag[1] = static_cast<int>(limit_us);
     fence_mbar_init();
   }
   __syncthreads();
   // phase 0 of `bar` never completes: the wait can only end by its time limit
-  const bool ok = mbar_wait<40>(smem_u32(&bar), 0, &abort_flag, limit_us);
+  const bool ok = mbar_wait<40>(smem_u32(&bar), 0, abort_flag);
   __syncthreads();
   if (threadIdx.x == 0) {
     result2[0] = ok ? 1 : 0;
-    result2[1] = abort_flag;
+    result2[1] = abort_flag[0];
   }
 }
 }  // namespace
