@@ -44,7 +44,8 @@ _lib_path = None
 
 
 def library_path() -> str:
-    return _lib_path or _build.LIB_PATH
+    """The build `load()` opens: `use_library()`'s choice, else $LT_INDEXER_LIB, else the in-tree release build."""
+    return _lib_path or os.environ.get("LT_INDEXER_LIB") or _build.LIB_PATH
 
 
 def use_library(path: Optional[str]) -> None:
