@@ -98,7 +98,7 @@ struct Layout {
   bool fused;
   // zeroed region
   size_t ctl, tail, hist, row_flag, block_flag, zero_end;
-  size_t smin, width, thr, fb_list, sample, gather_k, gather_scale, cand, scratch, total;
+  size_t smin, width, thr, fb_list, sample, gather_k, gather_scale, cand, scratch, fb_base, total;
   int cap, n_sample, sample_stride, sample_rank, fb_slots, n_blocks, generic_rows;
 };
 
@@ -191,9 +191,15 @@ Layout make_layout(bool fused, int T, int N, int topk, int causal_offset, const 
   off = align_up(off + static_cast<size_t>(T) * L.cap * 8);
   size_t slot_bytes = static_cast<size_t>(kRowsPerBlock) * N * 4;
   long long slots = static_cast<long long>(kFallbackScratchBudget / slot_bytes);
-  L.fb_slots = static_cast<int>(slots < 1 ? 1 : (slots > L.n_blocks ? L.n_blocks : slots));
+  const int own_slots = static_cast<int>(slots < 1 ? 1 : (slots > L.n_blocks ? L.n_blocks : slots));
   L.scratch = off;
-  off = align_up(off + static_cast<size_t>(L.fb_slots) * slot_bytes);
+  off = align_up(off + static_cast<size_t>(own_slots) * slot_bytes);
+  // The candidate buffers are dead once the final select has run, and the fallback's dense rows are only written
+  // after it: a fallback round uses the candidate region and the scratch behind it as one buffer, which makes the
+  // rounds (two launches each, all of them enqueued whether or not a row is flagged) fewer.
+  L.fb_base = L.cand;
+  const size_t fb_total_slots = (off - L.cand) / slot_bytes;
+  L.fb_slots = static_cast<int>(fb_total_slots > static_cast<size_t>(L.n_blocks) ? L.n_blocks : fb_total_slots);
   L.total = off;
   return L;
 }
@@ -327,7 +333,7 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
   int* fb_list = reinterpret_cast<int*>(ws + L.fb_list);
   float* sample = reinterpret_cast<float*>(ws + L.sample);
   uint2* cand = reinterpret_cast<uint2*>(ws + L.cand);
-  float* scratch = reinterpret_cast<float*>(ws + L.scratch);
+  float* scratch = reinterpret_cast<float*>(ws + L.fb_base);  // the fallback's dense rows (see make_layout)
 
   // 1. sample phase: score n_sample strided keys of the common prefix with the same tensor-core path
   //    (or, with a caller-provided sample, a dense copy of the keys at the given positions)
@@ -777,7 +783,7 @@ int lt_knn_topk(int dtype, const void* q, const void* x, int T, int N, int D, in
   int* fb_list = reinterpret_cast<int*>(ws + L.fb_list);
   float* sample = reinterpret_cast<float*>(ws + L.sample);
   uint2* cand = reinterpret_cast<uint2*>(ws + L.cand);
-  float* scratch = reinterpret_cast<float*>(ws + L.scratch);
+  float* scratch = reinterpret_cast<float*>(ws + L.fb_base);  // the fallback's dense rows (see make_layout)
 
   // 1. sample phase (paper Sec. 3.2 "Sampling": k-NN needs no history-based sample; a strided subsample of
   //    the corpus is used here), scored by the same tensor-core kernel
