@@ -293,6 +293,7 @@ def run_reference(args, rank: int):
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
         "config": {"workload": args.workload, "T": inp.T, "N": inp.N, "H": inp.H, "D": inp.D, "topk": inp.topk,
+                   "causal_offset": inp.causal_offset, "valid_pairs": inp.valid_pairs(), "parallelism": "replicas x1",
                    "note": "CPU oracle (numpy fp64 + full sort) on a bounded row sample of the workload"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
