@@ -2,7 +2,7 @@
 
 The acceptance rules decide whether a GPU result passes, so a mistake in them (a tolerance compared the wrong way
 round, `extra` and `missing` swapped, a skipped padding check) would make the index rule vacuous without any test
-failing.  Each rule is therefore driven with hand-made rows whose verdict is known from the rule's definition:
+failing.  Each rule is therefore driven with hand-made rows whose outcome is known from the rule's definition:
 legal boundary swaps must pass, every kind of illegal result must fail.  `indexer_scores`, the reference of every
 dense-score parity check, is compared value by value with the exact-rational brute force.
 """
