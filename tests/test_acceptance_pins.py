@@ -1,4 +1,4 @@
-"""Pins for the judge of every parity test (oracle/acceptance.py) and for the dense-score oracle.
+"""Pins for the arbiter of every parity test (oracle/acceptance.py) and for the dense-score oracle.
 
 The acceptance rules decide whether a GPU result passes, so a mistake in them (a tolerance compared the wrong way
 round, `extra` and `missing` swapped, a skipped padding check) would make the index rule vacuous without any test
