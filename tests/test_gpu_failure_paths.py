@@ -79,3 +79,12 @@ def test_row_strided_keys_give_the_dense_bits(name, T, N, topk, pitch):
     assert st[0] & lt.LT_STATUS_TIMEOUT == 0
     assert np.array_equal(out_idx.cpu().numpy(), want_idx)
     assert np.array_equal(out_score.cpu().numpy().view(np.uint32), want_score.view(np.uint32))
+    # the exact fallback reads the keys through the same pitch: force every row through it
+    tun = lt.Tunables(path=lt.LT_PATH_FUSED, cap_mult=1, sample_rank=1)
+    ws2 = lt.alloc_workspace(inp.dtype, inp.T, inp.N, inp.H, inp.D, inp.topk, tun)
+    out_idx.fill_(-7)
+    lt.lt_indexer_topk_strided(inp.dtype, q, w, wide[:, : inp.D], ks, inp.topk, inp.causal_offset, out_idx, out_score, ws2, tun)
+    st = lt.lt_read_status(ws2)
+    assert st[1] > 0, "this tunable set should send rows through the fallback"
+    assert np.array_equal(out_idx.cpu().numpy(), want_idx)
+    assert np.array_equal(out_score.cpu().numpy().view(np.uint32), want_score.view(np.uint32))
