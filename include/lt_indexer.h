@@ -89,8 +89,9 @@ typedef struct lt_tunables {
                         the paper reports in Sec. 4.2).  Default (0): max(12 topk, 16384) entries; an explicit
                         value is taken as given                                               */
   int sample_mult;   /* sample size k' = sample_mult * topk (paper Sec. 3.2: 3).  Default (0): max(3 topk,
-                        8192), but no more than 64 * (keys the sample is drawn from) / topk, which is
-                        what the default sample_rank needs; an explicit value is taken as given      */
+                        min(8192, keys the sample is drawn from / 32)), but no more than 64 * (keys the
+                        sample is drawn from) / topk, which is what the default sample_rank needs; an
+                        explicit value is taken as given                                           */
   int segment_tiles; /* key tiles (128 keys each) per work item (default 256)            */
   int grid;          /* CTAs of the scan kernel (default: number of SMs)                 */
   int sample_rank;   /* initial gate = lower edge of the bin holding the sample's r-th largest

@@ -152,7 +152,11 @@ Layout make_layout(bool fused, int T, int N, int topk, int causal_offset, const 
     // opposite case: 3k keys hold less than one of the row's top-k, the gate starts orders of magnitude too
     // loose and the candidate buffers overflow, so the sample is at least 8,192 keys (6 % of a 1M-key scan
     // at most).
-    if (want < 8192) want = 8192;
+    // ... but no more than 1/32 of the keys it is drawn from: over a 64K context 8,192 samples would be an eighth
+    // of the scan, while 2,048 still put a dozen top-k keys' worth of rank between the gate and the k-th score
+    long long floor_n = prefix / 32;
+    if (floor_n > 8192) floor_n = 8192;
+    if (want < floor_n) want = floor_n;
     long long enough = (64 * prefix + topk - 1) / topk;
     enough = (enough + kTileKeys - 1) / kTileKeys * kTileKeys;
     if (enough < want) want = enough;

@@ -107,7 +107,8 @@ def test_sample_plan_rank_keeps_misjudgement_below_1e6(lib):
         n_sample, stride, rank = binding.lt_indexer_sample_plan(N, topk, causal_offset)
         prefix = min(causal_offset + 1, N)
         enough = -(-(-(-64 * prefix // topk)) // 128) * 128  # 64 expected top-k keys in the sample, whole key tiles
-        assert n_sample == min(max(3 * topk, 8192), enough, prefix) and stride == prefix // n_sample and 1 <= rank <= topk
+        floor_n = min(8192, prefix // 32)  # at least 8192 samples, but never more than 1/32 of the prefix
+        assert n_sample == min(max(3 * topk, floor_n), enough, prefix) and stride == prefix // n_sample and 1 <= rank <= topk
         if rank < topk:
             # worst case for the tail: all topk of the row's best keys lie in the sampled prefix
             tail = hypergeom.sf(rank - 1, prefix, topk, n_sample)
