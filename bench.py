@@ -727,6 +727,8 @@ def main():
     ap.add_argument("--knn-sweep", action="store_true",
                     help="k-NN workloads: also time prefixes of the corpus (1M, 2M, 4M, ... vectors) x k in {128, 1024, 4096, 8192} "
                          "(the grid of the paper's retrieval benchmark) and add the table as 'sweep'")
+    ap.add_argument("--path", default="default", choices=["default", "abs"],
+                    help="abs: the alternative fp8 scan (LT_PATH_FUSED_ABS: |x| form of Eq. 1 with linear-term columns)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true",
                     help="default fp8_1m line only: skip the brief measurements of the other configurations and the next-row operations")
@@ -804,8 +806,11 @@ def main():
     q, w, k, ks = lt.to_device(inp)
     out_idx = torch.empty((inp.T, inp.topk), dtype=torch.int32, device="cuda")
     out_score = torch.empty((inp.T, inp.topk), dtype=torch.float32, device="cuda")
+    tun = lt.Tunables(path=lt.LT_PATH_FUSED_ABS) if args.path == "abs" else None
+    if tun is not None and (args.paged or sample_idx is not None):
+        raise SystemExit("--path abs is timed on the dense layout with the default sampler")
     if sample_idx is None:
-        ws = lt.alloc_workspace(inp.dtype, inp.T, inp.N, inp.H, inp.D, inp.topk)
+        ws = lt.alloc_workspace(inp.dtype, inp.T, inp.N, inp.H, inp.D, inp.topk, tun)
     else:
         ws = torch.empty(lt.lt_indexer_topk_sampled_workspace_bytes(inp.dtype, inp.T, inp.N, inp.H, inp.D, inp.topk,
                                                                     sample_idx.numel()), dtype=torch.uint8, device="cuda")
@@ -836,7 +841,7 @@ def main():
         if page_table is not None:
             lt.lt_indexer_topk_paged(inp.dtype, q_, w_, k_, ks_, page_table, inp.N, inp.topk, inp.causal_offset, idx_, score_, ws)
         elif sample_idx is None:
-            lt.lt_indexer_topk_ex(inp.dtype, q_, w_, k_, ks_, inp.topk, inp.causal_offset, idx_, score_, ws)
+            lt.lt_indexer_topk_ex(inp.dtype, q_, w_, k_, ks_, inp.topk, inp.causal_offset, idx_, score_, ws, tun)
         else:
             lt.lt_indexer_topk_sampled(inp.dtype, q_, w_, k_, ks_, inp.topk, inp.causal_offset, sample_idx, idx_, score_, ws)
 
@@ -956,7 +961,8 @@ def main():
     scan_ms = statistics.mean(p[2] for p in phase_ms)
     achieved = flops / (scan_ms * 1e-3) / 1e12
     roofline = {
-        "bound": "tensor", "kernel": "scan_kernel (fused score + filter)", "achieved": achieved, "peak": peak_tflops,
+        "bound": "tensor", "kernel": "scan_fp8_kernel (alternative |x| form)" if tun is not None else "scan_kernel (fused score + filter)",
+        "achieved": achieved, "peak": peak_tflops,
         "unit": "TFLOP/s", "frac": achieved / peak_tflops, "peak_kind": f"of {peak_kind} (bf16 burst x {2 if fp8 else 1})",
         "frac_of_nominal": achieved / (NOMINAL_FP8_TFLOPS if fp8 else NOMINAL_BF16_TFLOPS),
         # context: the same kernel against the power-capped (seconds-long) cuBLAS figure; the timed loop of
@@ -978,7 +984,8 @@ def main():
         "config": {"workload": args.workload, "T": inp.T, "N": inp.N, "H": inp.H, "D": inp.D, "topk": inp.topk,
                    "causal_offset": inp.causal_offset, "valid_pairs": pairs, "parallelism": f"replicas x{world}",
                    "l2": "flushed between timed iterations (256 MiB write)", "workspace_bytes": int(ws.numel()),
-                   "key_layout": "paged (64-key pages, random order)" if page_table is not None else "dense"},
+                   "key_layout": "paged (64-key pages, random order)" if page_table is not None else "dense",
+                   "path": args.path},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps,
@@ -1003,7 +1010,8 @@ def main():
     if args.aux:
         line["aux"] = time_aux_ops(torch, lt, out_idx, inp, peaks["hbm_gbs"], peak_kind)
 
-    default_line = (args.workload == "fp8_1m" and not args.rows and page_table is None and sample_idx is None and world == 1)
+    default_line = (args.workload == "fp8_1m" and not args.rows and page_table is None and sample_idx is None and world == 1
+                    and tun is None)
     if default_line and not args.no_extras:
         # the other four configurations and the "next" operations, a few timed steps each, in the same process
         del dev2, outs2, h_outs2, host

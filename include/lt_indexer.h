@@ -78,6 +78,12 @@ extern "C" {
 #define LT_PATH_AUTO 0    /* fused tensor-core path when the shape allows it, else generic */
 #define LT_PATH_FUSED 1   /* fused tcgen05 path; LT_ERR_UNSUPPORTED if the shape does not fit */
 #define LT_PATH_GENERIC 2 /* generic SIMT scoring + full-row select (any H, D, dtype)      */
+#define LT_PATH_FUSED_ABS 3 /* fp8 only: an alternative fused tensor-core scan that evaluates Eq. 1 as
+                               sum_h (w_h / 2) |x_h| + (1/2) (sum_h w_h q_h) . k (ReLU(x) = (x + |x|) / 2), the linear
+                               term riding on the tensor core as five e4m3-split accumulator columns per query.
+                               Exact like the default (its own scores, lt_indexer_scores with the same path, are
+                               within the same tolerance of Eq. 1 and ranked bit-exactly), but slower as measured;
+                               kept as a documented alternative.  LT_ERR_UNSUPPORTED for other dtypes / shapes     */
 
 /*
  * Tunables.  None of them may change any output bit; they trade memory and speed.

@@ -16,7 +16,7 @@ import torch
 from . import build as _build
 
 LT_DTYPE_F32, LT_DTYPE_BF16, LT_DTYPE_E4M3 = 0, 1, 2
-LT_PATH_AUTO, LT_PATH_FUSED, LT_PATH_GENERIC = 0, 1, 2
+LT_PATH_AUTO, LT_PATH_FUSED, LT_PATH_GENERIC, LT_PATH_FUSED_ABS = 0, 1, 2, 3
 LT_OK = 0
 LT_STATUS_TIMEOUT, LT_STATUS_FALLBACK, LT_STATUS_BOUNDS = 1, 2, 4
 LT_DEBUG_SKIP_ONE_KTILE = 1

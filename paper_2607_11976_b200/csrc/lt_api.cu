@@ -92,23 +92,31 @@ int check_problem(int dtype, const void* q, const float* w, const void* k, const
 bool use_fused(const Tun& tun, int dtype, int H, int D) {
   return tun.path != LT_PATH_GENERIC && scan_mma_supported(dtype, H, D);
 }
+// the alternative fp8 scan (|x| form with linear-term columns, 6-row query blocks) was asked for and applies
+bool use_abs_form(const Tun& tun, int dtype, int H, int D) {
+  return tun.path == LT_PATH_FUSED_ABS && dtype == LT_DTYPE_E4M3 && scan_mma_supported(dtype, H, D);
+}
 
 // ---- workspace layout ------------------------------------------------------------------------
 struct Layout {
   bool fused;
   // zeroed region
   size_t ctl, tail, hist, row_flag, block_flag, zero_end;
-  size_t smin, width, thr, fb_list, sample, gather_k, gather_scale, cand, scratch, fb_base, total;
+  size_t smin, width, thr, fb_list, lin_q, lin_scale, sample, gather_k, gather_scale, cand, scratch, fb_base, total;
   int cap, n_sample, sample_stride, sample_rank, fb_slots, n_blocks, generic_rows;
+  int rpb;        // rows of one scan block = rows of one fallback block
+  bool abs_form;  // the alternative fp8 scan: linear-term rows live in the workspace
 };
 
 // n_given > 0: the caller provides that many sample positions (lt_indexer_topk_sampled); their keys are
 // gathered into a dense buffer of the workspace (key_row_bytes each) and scored from there.
 // gather_default: the default strided sample is gathered too (paged key cache: a strided view cannot reach it).
 Layout make_layout(bool fused, int T, int N, int topk, int causal_offset, const Tun& tun, int n_given = 0,
-                   int key_row_bytes = 0, bool gather_default = false) {
+                   int key_row_bytes = 0, bool gather_default = false, bool abs_form = false) {
   Layout L{};
   L.fused = fused;
+  L.abs_form = fused && abs_form;
+  L.rpb = L.abs_form ? kRowsPerBlockFp8 : kRowsPerBlock;
   size_t off = 0;
   L.ctl = off;
   off = align_up(off + sizeof(Control));
@@ -121,7 +129,7 @@ Layout make_layout(bool fused, int T, int N, int topk, int causal_offset, const 
     L.total = off;
     return L;
   }
-  L.n_blocks = (T + kRowsPerBlock - 1) / kRowsPerBlock;
+  L.n_blocks = (T + L.rpb - 1) / L.rpb;
   L.tail = off;
   off = align_up(off + static_cast<size_t>(T) * 4);
   L.hist = off;
@@ -139,6 +147,11 @@ Layout make_layout(bool fused, int T, int N, int topk, int causal_offset, const 
   off = align_up(off + static_cast<size_t>(T) * 4);
   L.fb_list = off;
   off = align_up(off + static_cast<size_t>(L.n_blocks) * 4);
+  // alternative fp8 scan: operand rows and scales of the linear part of Eq. 1 (lt_scan_fp8.cu)
+  L.lin_q = off;
+  if (L.abs_form) off = align_up(off + lin_q_bytes(T));
+  L.lin_scale = off;
+  if (L.abs_form) off = align_up(off + lin_scale_bytes(T));
   // sample: keys every chunk row can see, i.e. positions 0 .. causal_offset, strided
   long long prefix = static_cast<long long>(causal_offset) + 1;
   if (prefix > N) prefix = N;
@@ -193,7 +206,7 @@ Layout make_layout(bool fused, int T, int N, int topk, int causal_offset, const 
   L.cap = static_cast<int>(cap > N ? N : cap);
   L.cand = off;
   off = align_up(off + static_cast<size_t>(T) * L.cap * 8);
-  size_t slot_bytes = static_cast<size_t>(kRowsPerBlock) * N * 4;
+  size_t slot_bytes = static_cast<size_t>(L.rpb) * N * 4;
   long long slots = static_cast<long long>(kFallbackScratchBudget / slot_bytes);
   const int own_slots = static_cast<int>(slots < 1 ? 1 : (slots > L.n_blocks ? L.n_blocks : slots));
   L.scratch = off;
@@ -243,6 +256,13 @@ int pick_seg_tiles(const Tun& tun, int n_keys, int n_blocks, int grid) {
     }
   }
   return best;
+}
+
+// the default scan kernels, or the alternative fp8 scan, behind the same parameter block
+cudaError_t launch_scan(bool abs_form, int dtype, int mode, const void* q, int T, const void* k, long long n_keys_view,
+                        long long key_pitch_elems, const ScanParams& p, int grid, cudaStream_t stream) {
+  if (abs_form) return launch_scan_fp8(mode, q, T, k, n_keys_view, key_pitch_elems, p, grid, stream);
+  return launch_scan_mma(dtype, mode, q, T, k, n_keys_view, key_pitch_elems, p, grid, stream);
 }
 
 // Control block for entry points that have no workspace (lt_indexer_scores).
@@ -308,12 +328,14 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
   if (out_idx == nullptr || topk <= 0 || topk > N || topk > LT_MAX_TOPK) return LT_ERR_INVALID_ARG;
   const Tun tun = resolve_tunables(tunables);
   const bool fused = use_fused(tun, dtype, H, D);
-  if (tun.path == LT_PATH_FUSED && !fused) return LT_ERR_UNSUPPORTED;
+  if ((tun.path == LT_PATH_FUSED || tun.path == LT_PATH_FUSED_ABS) && !fused) return LT_ERR_UNSUPPORTED;
   const int key_row_bytes = static_cast<int>(static_cast<size_t>(D) * elem_bytes(dtype));
   const bool paged = page_table != nullptr;
   if (paged && !fused) return LT_ERR_UNSUPPORTED;
   if (key_pitch != D && (!fused || paged || n_given > 0)) return LT_ERR_UNSUPPORTED;
-  const Layout L = make_layout(fused, T, N, topk, causal_offset, tun, n_given, key_row_bytes, paged);
+  const bool abs_form = use_abs_form(tun, dtype, H, D);
+  if (tun.path == LT_PATH_FUSED_ABS && !abs_form) return LT_ERR_UNSUPPORTED;
+  const Layout L = make_layout(fused, T, N, topk, causal_offset, tun, n_given, key_row_bytes, paged, abs_form);
   const long long key_rows = paged ? pool_rows : N;  // rows the key tensor map covers
   if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) != 0 || workspace_bytes < L.total)
     return LT_ERR_WORKSPACE;
@@ -338,10 +360,15 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
   float* sample = reinterpret_cast<float*>(ws + L.sample);
   uint2* cand = reinterpret_cast<uint2*>(ws + L.cand);
   float* scratch = reinterpret_cast<float*>(ws + L.fb_base);  // the fallback's dense rows (see make_layout)
+  void* lin_q = abs_form ? ws + L.lin_q : nullptr;
+  float* lin_scale = abs_form ? reinterpret_cast<float*>(ws + L.lin_scale) : nullptr;
+
+  // 0. alternative fp8 scan: the linear part of Eq. 1 as extra operand rows of every query (used by all scans below)
+  mark_phase(0, stream);
+  if (abs_form) LT_LAUNCH(launch_lin_terms(q, w, T, lin_q, lin_scale, stream));
 
   // 1. sample phase: score n_sample strided keys of the common prefix with the same tensor-core path
   //    (or, with a caller-provided sample, a dense copy of the keys at the given positions)
-  mark_phase(0, stream);
   const void* sample_keys = k;
   const float* sample_scale = k_scale;
   long long sample_pitch = static_cast<long long>(L.sample_stride) * key_pitch;
@@ -371,8 +398,10 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
     p.topk = topk;
     p.dump = sample;
     p.dump_ld = L.n_sample;
+    p.lin_q = lin_q;
+    p.lin_scale = lin_scale;
     p.ctl = ctl;
-    LT_LAUNCH(launch_scan_mma(dtype, kModeDump, q, T, sample_keys, L.n_sample, sample_pitch, p, grid, stream));
+    LT_LAUNCH(launch_scan(abs_form, dtype, kModeDump, q, T, sample_keys, L.n_sample, sample_pitch, p, grid, stream));
   }
   mark_phase(1, stream);
   LT_LAUNCH(launch_sample_stats(sample, T, L.n_sample, L.sample_rank, smin, width, thr, stream));
@@ -404,8 +433,10 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
     p.n_pages = n_pages;
     p.pool_pages = pool_rows / kPageKeys;
     p.debug_flags = tun.debug_flags;
+    p.lin_q = lin_q;
+    p.lin_scale = lin_scale;
     p.ctl = ctl;
-    LT_LAUNCH(launch_scan_mma(dtype, kModeFilter, q, T, k, key_rows, key_pitch, p, grid, stream));
+    LT_LAUNCH(launch_scan(abs_form, dtype, kModeFilter, q, T, k, key_rows, key_pitch, p, grid, stream));
   }
 
   // 3. final select over the survivors; rows it cannot finish exactly are flagged
@@ -427,6 +458,7 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
     p.row_flag = row_flag;
     p.block_flag = block_flag;
     p.fb_list = fb_list;
+    p.rows_per_block = L.rpb;
     p.ctl = ctl;
     LT_LAUNCH(launch_final_select(p, stream));
   }
@@ -458,12 +490,15 @@ int topk_impl(int dtype, const void* q, const float* w, const void* k, const flo
     p.page_table = page_table;
     p.n_pages = n_pages;
     p.pool_pages = pool_rows / kPageKeys;
+    p.lin_q = lin_q;
+    p.lin_scale = lin_scale;
     p.ctl = ctl;
-    LT_LAUNCH(launch_scan_mma(dtype, kModeDump, q, T, k, key_rows, key_pitch, p, grid, stream));
+    LT_LAUNCH(launch_scan(abs_form, dtype, kModeDump, q, T, k, key_rows, key_pitch, p, grid, stream));
     SelectRowsParams sp{};
     sp.scores = scratch;
     sp.ld = N;
-    sp.n_blocks = L.fb_slots * kRowsPerBlock;
+    sp.n_blocks = L.fb_slots * L.rpb;
+    sp.rows_per_block = L.rpb;
     sp.T = T;
     sp.N = N;
     sp.topk = topk;
@@ -542,7 +577,7 @@ size_t lt_indexer_topk_workspace_bytes(int dtype, int T, int N, int H, int D, in
     return 0;
   const Tun tun = resolve_tunables(tunables);
   // the sample can never be larger with a different causal_offset than with the whole context visible
-  return make_layout(use_fused(tun, dtype, H, D), T, N, topk, N - 1, tun).total;
+  return make_layout(use_fused(tun, dtype, H, D), T, N, topk, N - 1, tun, 0, 0, false, use_abs_form(tun, dtype, H, D)).total;
 }
 
 int lt_indexer_topk_sampled(int dtype, const void* q, const float* w, const void* k, const float* k_scale, int T, int N, int H,
@@ -561,7 +596,7 @@ size_t lt_indexer_topk_sampled_workspace_bytes(int dtype, int T, int N, int H, i
     return 0;
   const Tun tun = resolve_tunables(tunables);
   return make_layout(use_fused(tun, dtype, H, D), T, N, topk, N - 1, tun, n_sample,
-                     static_cast<int>(static_cast<size_t>(D) * elem_bytes(dtype))).total;
+                     static_cast<int>(static_cast<size_t>(D) * elem_bytes(dtype)), false, use_abs_form(tun, dtype, H, D)).total;
 }
 
 int lt_indexer_topk_paged(int dtype, const void* q, const float* w, const void* k_pool, const float* k_scale_pool,
@@ -581,7 +616,8 @@ size_t lt_indexer_topk_paged_workspace_bytes(int dtype, int T, int N, int H, int
     return 0;
   const Tun tun = resolve_tunables(tunables);
   if (!use_fused(tun, dtype, H, D)) return 0;
-  return make_layout(true, T, N, topk, N - 1, tun, 0, static_cast<int>(static_cast<size_t>(D) * elem_bytes(dtype)), true).total;
+  return make_layout(true, T, N, topk, N - 1, tun, 0, static_cast<int>(static_cast<size_t>(D) * elem_bytes(dtype)), true,
+                     use_abs_form(tun, dtype, H, D)).total;
 }
 
 size_t lt_topk_frequent_workspace_bytes(int N) {
@@ -688,11 +724,22 @@ int lt_indexer_scores(int dtype, const void* q, const float* w, const void* k, c
   // run_unfused with topk == 0 only dumps; rows are written straight to the caller's matrix
   const float* kk = k_scale;
   int rows = row_end - row_begin;
+  const bool abs_form = use_abs_form(tun, dtype, H, D);
+  if (path == LT_PATH_FUSED_ABS && !abs_form) return LT_ERR_UNSUPPORTED;
   if (mma) {
     // the scan kernel addresses dump rows relative to row_begin
     ScanParams p{};
     p.wait_limit_us = tun.wait_limit_us;
     const int grid = sm_count();
+    void* lin = nullptr;
+    if (abs_form) {
+      // linear terms of all rows: a stream-ordered temporary (this entry point has no workspace)
+      const size_t qb = align_up(lin_q_bytes(T));
+      LT_CUDA(cudaMallocAsync(&lin, qb + lin_scale_bytes(T), stream));
+      p.lin_q = lin;
+      p.lin_scale = reinterpret_cast<float*>(static_cast<uint8_t*>(lin) + qb);
+      LT_LAUNCH(launch_lin_terms(q, w, T, lin, const_cast<float*>(p.lin_scale), stream));
+    }
     p.w = w;
     p.k_scale = kk;
     p.ks_stride = 1;
@@ -702,11 +749,13 @@ int lt_indexer_scores(int dtype, const void* q, const float* w, const void* k, c
     p.n_keys = N;
     p.causal_offset = causal_offset;
     p.skip_masked_tiles = 0;
-    p.seg_tiles = pick_seg_tiles(tun, N, (rows + kRowsPerBlock - 1) / kRowsPerBlock, grid);
+    const int rpb = abs_form ? kRowsPerBlockFp8 : kRowsPerBlock;
+    p.seg_tiles = pick_seg_tiles(tun, N, (rows + rpb - 1) / rpb, grid);
     p.dump = out_scores;
     p.dump_ld = N;
     p.ctl = ctl;
-    LT_LAUNCH(launch_scan_mma(dtype, kModeDump, q, T, k, N, D, p, grid, stream));
+    LT_LAUNCH(launch_scan(abs_form, dtype, kModeDump, q, T, k, N, D, p, grid, stream));
+    if (lin != nullptr) LT_CUDA(cudaFreeAsync(lin, stream));
   } else {
     LT_LAUNCH(launch_simt_scores(dtype, q, w, k, kk, T, N, H, D, causal_offset, row_begin, row_end, out_scores, N, stream));
   }
@@ -851,6 +900,7 @@ int lt_knn_topk(int dtype, const void* q, const void* x, int T, int N, int D, in
     p.row_flag = row_flag;
     p.block_flag = block_flag;
     p.fb_list = fb_list;
+    p.rows_per_block = kRowsPerBlock;
     p.ctl = ctl;
     LT_LAUNCH(launch_final_select(p, stream));
   }
@@ -906,6 +956,7 @@ int lt_unfused_topk(int dtype, const void* q, const float* w, const void* k, con
   tun.path = path;
   const bool mma = use_fused(tun, dtype, H, D);
   if (path == LT_PATH_FUSED && !mma) return LT_ERR_UNSUPPORTED;
+  if (path == LT_PATH_FUSED_ABS) return LT_ERR_UNSUPPORTED;  // the decoupled baseline scores with the default kernels
   // the first 256 bytes of score_buf hold the status block (readable with lt_read_status)
   if (score_buf_bytes < kAlign + static_cast<size_t>(N) * 4) return LT_ERR_WORKSPACE;
   long long rows = static_cast<long long>((score_buf_bytes - kAlign) / (static_cast<size_t>(N) * 4));

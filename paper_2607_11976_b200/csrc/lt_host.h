@@ -11,7 +11,10 @@ namespace lt {
 
 constexpr int kModeFilter = 0;
 constexpr int kModeDump = 1;
-constexpr int kRowsPerBlock = 8;  // query rows one scan CTA keeps resident
+constexpr int kRowsPerBlock = 8;     // query rows one scan CTA (and one k-NN fallback block) keeps resident
+constexpr int kRowsPerBlockFp8 = 6;  // ... of the alternative fp8 scan (LT_PATH_FUSED_ABS, lt_scan_fp8.cu)
+constexpr int kLinTerms = 5;         // e4m3 terms of the linear part of a query (alternative fp8 scan)
+constexpr int kLinScaleStride = 8;   // floats per row of the linear-term scale table
 
 // Parameters of the tensor-core scan kernel (lt_scan_mma.cu).
 struct ScanParams {
@@ -49,11 +52,22 @@ struct ScanParams {
   long long pool_pages;    // pages of the pool behind page_table (bounds checks of the debug build)
   unsigned int wait_limit_us;  // bound of every device-side wait (0 is replaced by the default at launch)
   int debug_flags;         // LT_DEBUG_* test hooks (filter mode only)
+  // alternative fp8 scan only: the linear part of Eq. 1 prepared by launch_lin_terms
+  const void* lin_q;       // [T][kLinTerms][128] e4m3 codes
+  const float* lin_scale;  // [T][kLinScaleStride], the first kLinTerms entries of a row are used
   Control* ctl;
 };
 constexpr int kPageKeys = 64;  // keys per page of a paged key cache
 
 bool scan_mma_supported(int dtype, int H, int D);
+// ---- lt_scan_fp8.cu: the alternative fp8 scan (|x| form of Eq. 1 with linear-term columns) ------------
+// bytes of the linear-term operand rows / of the scale table of T query rows
+inline size_t lin_q_bytes(int T) { return static_cast<size_t>(T) * kLinTerms * 128; }
+inline size_t lin_scale_bytes(int T) { return static_cast<size_t>(T) * kLinScaleStride * 4; }
+// pre-pass: q [T][64][128] e4m3, w [T][64] -> lin_q, lin_scale
+cudaError_t launch_lin_terms(const void* q, const float* w, int T, void* lin_q, float* lin_scale, cudaStream_t stream);
+cudaError_t launch_scan_fp8(int mode, const void* q, int T, const void* k, long long n_keys_view, long long key_pitch_elems,
+                            const ScanParams& p, int grid, cudaStream_t stream);
 
 // One warp waits, with the bounded wait every scan kernel uses, on a barrier nobody arrives at:
 // result2[0] = what the wait returned (0 = gave up), result2[1] = the abort flag it left behind.
@@ -115,15 +129,16 @@ struct FinalSelectParams {
   int32_t* out_idx;
   float* out_score;
   unsigned char* row_flag;    // [T] 1 = needs the fallback
-  unsigned int* block_flag;   // [ceil(T/8)]
-  int* fb_list;               // [ceil(T/8)]
+  unsigned int* block_flag;   // [ceil(T / rows_per_block)]
+  int* fb_list;               // [ceil(T / rows_per_block)]
+  int rows_per_block;         // rows of one fallback block (the scan kernel's query block)
   Control* ctl;
 };
 cudaError_t launch_final_select(const FinalSelectParams& p, cudaStream_t stream);
 
 // Full-row exact select over dense scores.  Direct mode: block b handles row row_begin + b whose
-// scores start at scores + b * ld.  Fallback mode (fb_list != null): block b handles row
-// fb_list[fb_round_base + b / 8] * 8 + b % 8 if that row is flagged; scores at scores + b * ld.
+// scores start at scores + b * ld.  Fallback mode (fb_list != null), R = rows_per_block: block b handles row
+// fb_list[fb_round_base + b / R] * R + b % R if that row is flagged; scores at scores + b * ld.
 struct SelectRowsParams {
   const float* scores;
   long long ld;
@@ -135,6 +150,7 @@ struct SelectRowsParams {
   const int* fb_list;
   const int* fb_blocks;
   int fb_round_base;
+  int rows_per_block;
   const unsigned char* row_flag;
   Control* ctl;
 };

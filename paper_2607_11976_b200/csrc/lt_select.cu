@@ -578,9 +578,9 @@ __global__ void __launch_bounds__(kFinalThreads) final_select_kernel(const Final
     p.row_flag[t] = 1;
     atomicOr(&p.ctl->status, LT_STATUS_FALLBACK);
     atomicAdd(&p.ctl->fb_rows, 1);
-    if (atomicExch(p.block_flag + t / kRowsPerBlock, 1u) == 0u) {
+    if (atomicExch(p.block_flag + t / p.rows_per_block, 1u) == 0u) {
       int pos = atomicAdd(&p.ctl->fb_blocks, 1);
-      p.fb_list[pos] = t / kRowsPerBlock;
+      p.fb_list[pos] = t / p.rows_per_block;
     }
   }
 }
@@ -596,9 +596,9 @@ __global__ void __launch_bounds__(kSelThreads) select_rows_kernel(const SelectRo
   __shared__ unsigned int warp_cnt[32];
   int t;
   if (p.fb_list != nullptr) {
-    int j = p.fb_round_base + blockIdx.x / kRowsPerBlock;
+    int j = p.fb_round_base + blockIdx.x / p.rows_per_block;
     if (j >= *p.fb_blocks) return;
-    t = p.fb_list[j] * kRowsPerBlock + blockIdx.x % kRowsPerBlock;
+    t = p.fb_list[j] * p.rows_per_block + blockIdx.x % p.rows_per_block;
     if (t >= p.T || !p.row_flag[t]) return;
   } else {
     t = p.row_begin + blockIdx.x;
