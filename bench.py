@@ -121,7 +121,7 @@ class ClockSampler:
 
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+              "clocks_event_reasons.sw_power_cap,power.limit")
 
     def __init__(self, gpu_index: int):
         self.gpu_index = gpu_index
@@ -152,7 +152,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, smax, power, reasons = [], [], [], set()
+        sm, smax, power, limit, reasons = [], [], [], [], set()
         for line in self.lines:
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 7:
@@ -163,13 +163,19 @@ class ClockSampler:
                 power.append(float(parts[2]))
             except ValueError:
                 continue
+            try:
+                limit.append(float(parts[7]))
+            except (ValueError, IndexError):
+                pass
             for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[3:7]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         # the busiest samples are the ones under load
         loaded = [c for c, p in zip(sm, power) if power and p >= 0.6 * max(power)] or sm
+        loaded_w = [p for p in power if p >= 0.6 * max(power)] or power
         return {"sm_mhz": statistics.median(loaded) if loaded else None, "sm_max_mhz": max(smax) if smax else None,
-                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+                "power_w": statistics.median(loaded_w) if loaded_w else None, "power_w_max": max(power) if power else None,
+                "power_limit_w": max(limit) if limit else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
 def max_over_ranks(value: float, world: int, device) -> float:
