@@ -121,7 +121,7 @@ class ClockSampler:
 
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap,power.limit")
+              "clocks_event_reasons.sw_power_cap,power.limit,power.draw.instant")
 
     def __init__(self, gpu_index: int):
         self.gpu_index = gpu_index
@@ -130,9 +130,16 @@ class ClockSampler:
         self.thread = None
 
     def start(self):
+        fields = self.FIELDS
+        try:
+            probe = subprocess.run(["nvidia-smi", f"--id={self.gpu_index}", "--query-gpu=power.draw.instant", "--format=csv,noheader,nounits"],
+                                   capture_output=True, text=True, timeout=20)
+            float(probe.stdout.strip().splitlines()[0])
+        except (OSError, ValueError, IndexError, subprocess.TimeoutExpired):
+            fields = fields.replace(",power.draw.instant", "")  # older drivers: the averaged reading only
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={fields}", "--format=csv,noheader,nounits", "-lms", "100"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -165,6 +172,7 @@ class ClockSampler:
                 continue
             try:
                 limit.append(float(parts[7]))
+                power[-1] = float(parts[8])  # the instantaneous reading where the driver has one (power.draw averages over ~1 s)
             except (ValueError, IndexError):
                 pass
             for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[3:7]):
