@@ -22,6 +22,8 @@ def run_topk(inp, tunables=None, entry="ex"):
         lt.lt_indexer_topk_ex(inp.dtype, q, w, k, ks, inp.topk, inp.causal_offset, out_idx, out_score, ws, tunables)
         status = lt.lt_read_status(ws)
     torch.cuda.synchronize()
+    # only the bounds-checking build can set this bit (the whole suite also runs against it: LT_INDEXER_LIB)
+    assert status[0] & lt.LT_STATUS_BOUNDS == 0, "an index check of the bounds-checking build failed"
     return out_idx.cpu().numpy(), out_score.cpu().numpy(), status
 
 
@@ -32,6 +34,7 @@ def run_unfused(inp, rows_per_pass=64, path=lt.LT_PATH_AUTO):
     buf = torch.empty(256 + rows_per_pass * inp.N * 4, dtype=torch.uint8, device="cuda")
     lt.lt_unfused_topk(inp.dtype, q, w, k, ks, inp.topk, inp.causal_offset, out_idx, out_score, buf, path)
     status = lt.lt_read_status(buf)
+    assert status[0] & lt.LT_STATUS_BOUNDS == 0, "an index check of the bounds-checking build failed"
     return out_idx.cpu().numpy(), out_score.cpu().numpy(), status
 
 
