@@ -281,6 +281,42 @@ def test_random_shapes_fused_path():
         assert_own_scores_rule(inp, idx, score, dumped, range(T))
 
 
+def test_soak_random_problems_with_random_tunables():
+    """A wider seeded sweep than the test above: eight recipes, chunks of 1 - 400 rows, up to 600,000 keys, any causal
+    offset, k up to 4096, random capacity / sample size / sample rank / work-item length / grid.  The arbiter is the
+    library's own dense dump (own-scores rule on every row, bit for bit), so a problem costs a fraction of a second.
+    LT_SOAK_PROBLEMS sets how many problems are drawn (default 24; 861 were run once, also against the bounds-checking
+    build, without a failure) and LT_SOAK_SEED which sequence."""
+    import os
+    rng = np.random.default_rng(int(os.environ.get("LT_SOAK_SEED", "1")))
+    names = ["dsa_bf16", "fp8_ar1", "hot_fp8", "adv_ties", "adv_planted", "adv_cluster", "adv_ties_exact", "fp8_1m"]
+    for _ in range(int(os.environ.get("LT_SOAK_PROBLEMS", "24"))):
+        name = names[int(rng.integers(0, len(names)))]
+        big = rng.random() < 0.2
+        T = int(rng.integers(1, 120 if big else 400))
+        N = int(rng.integers(T + 64, 600000 if big else 60000))
+        topk = int(rng.integers(1, min(N - T, 4096) + 1))
+        co = int(rng.integers(0, N - T + 1)) if rng.random() < 0.5 else None
+        r = rng.random()
+        if r < 0.25:
+            tun = lt.Tunables(path=lt.LT_PATH_FUSED, sample_mult=int(rng.integers(1, 8)), cap_mult=int(rng.integers(2, 16)))
+        elif r < 0.4:
+            tun = lt.Tunables(path=lt.LT_PATH_FUSED, sample_rank=int(rng.integers(1, 50)))
+        elif r < 0.5:
+            tun = lt.Tunables(path=lt.LT_PATH_FUSED, segment_tiles=int(rng.integers(1, 64)), grid=int(rng.integers(1, 149)))
+        else:
+            tun = lt.Tunables(path=lt.LT_PATH_FUSED)
+        inp = make_config(name, T=T, N=N, topk=topk, causal_offset=co, seed=int(rng.integers(0, 1 << 30)))
+        what = (name, T, N, topk, co, tun.cap_mult, tun.sample_mult, tun.sample_rank, tun.segment_tiles, tun.grid)
+        idx, score, status = run_topk(inp, tun)
+        assert status[0] & lt.LT_STATUS_TIMEOUT == 0, what
+        dumped = dump_scores(inp, 0, T, lt.LT_PATH_FUSED)
+        try:
+            assert_own_scores_rule(inp, idx, score, dumped, range(T))
+        except AssertionError as e:
+            raise AssertionError(f"{what}: {e}") from None
+
+
 @pytest.mark.parametrize("name", ["dsa_bf16", "fp8_ar1", "adv_ties_exact"])
 def test_final_select_branches(name):
     """Output sizes on both sides of the final select's branch points (radix sort of 512 .. 4096 gathered candidates,
