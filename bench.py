@@ -116,6 +116,47 @@ def measure_fp8_gemm(torch, n: int = 8192, sustained_s: float = 2.0):
         return {"unavailable": f"{type(exc).__name__}: {exc}"[:160]}
 
 
+def measure_umma_stream(torch, lt, gpu_index: int, seconds: float = 3.0):
+    """The library's bare FP8 UMMA stream (lt_debug_umma_stream: tcgen05.mma kind::f8f6f4 tiles of the scan's shape on
+    operands resident in shared memory, no TMA, no epilogue), one CTA per SM and as CTA pairs, each launched back to back
+    for `seconds` with the SM clock and the board power sampled: the tensor ceiling of this board at the power it is
+    granted.  Context for the tensor roofline; `roofline.peak` stays the measured bf16 figure x the nominal ratio."""
+    out = {}
+    try:
+        n_sm = torch.cuda.get_device_properties(0).multi_processor_count
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        iters, per_block = 4000, 20
+        for name, pair in (("single", False), ("pair", True)):
+            grid = n_sm & ~1 if pair else n_sm
+            flops = grid * iters * 16777216.0
+            for _ in range(3):
+                lt.lt_debug_umma_stream(pair, iters, status)
+            torch.cuda.synchronize()
+            sampler = ClockSampler(gpu_index)
+            sampler.start()
+            t0 = time.time()
+            ms_blocks = []
+            while time.time() - t0 < seconds:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(per_block):
+                    lt.lt_debug_umma_stream(pair, iters, status)
+                e1.record()
+                e1.synchronize()
+                ms_blocks.append(e0.elapsed_time(e1) / per_block)
+            clocks = sampler.stop()
+            tail = ms_blocks[len(ms_blocks) // 2:]  # the steady state: second half of the run
+            out[name] = {"tflops": flops / (statistics.median(tail) * 1e-3) / 1e12,
+                         "tflops_first_block": flops / (ms_blocks[0] * 1e-3) / 1e12,
+                         "sm_mhz": clocks.get("sm_mhz"), "power_w": clocks.get("power_w"), "reasons": clocks.get("reasons")}
+        out["status_bits"] = int(status.item())
+        out["how"] = (f"{iters} iterations x 8 UMMAs (M128 N256 K32, e4m3) per CTA and launch, launches back to back for "
+                      f"{seconds:.0f} s per form; tflops = median of the second half")
+    except Exception as exc:  # noqa: BLE001 - context figure only
+        return {"unavailable": f"{type(exc).__name__}: {exc}"[:160]}
+    return out
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
 
@@ -1020,6 +1061,11 @@ def main():
             g["frac_of_burst"] = achieved / g["burst_tflops"]
             g["frac_of_sustained"] = achieved / g["sustained_tflops"]
         roofline["fp8_gemm_measured"] = g
+        if not args.no_extras:
+            u = measure_umma_stream(torch, lt, local_rank)
+            if "single" in u:
+                u["frac_of_single"] = achieved / u["single"]["tflops"]
+            roofline["fp8_umma_stream_measured"] = u
 
     if args.aux:
         line["aux"] = time_aux_ops(torch, lt, out_idx, inp, peaks["hbm_gbs"], peak_kind)

@@ -352,6 +352,21 @@ int lt_read_status_static(int* status8_host, void* stream);
 int lt_debug_wait_timeout(int limit_us, int* result2_device, void* stream);
 
 /*
+ * Measurement aid (no counterpart in the paper; used by the benchmark): a bare FP8 tensor-core stream.  One
+ * launch of one CTA per SM; every CTA issues `iters` x 8 tcgen05.mma kind::f8f6f4 instructions of the scan's tile
+ * shape (128 keys x 256 (query, head) columns x 32 bytes; 2 x 128 x 256 x 128 x 2 flops per SM and iteration) on
+ * e4m3 operands that stay in shared memory: no TMA, no epilogue.  FLOPs of a launch = SMs x iters x 16,777,216.
+ * What it sustains is the tensor ceiling of the board at the clocks and power it is granted, against which the
+ * scan's roofline fraction can be read.
+ *   pair           0: cta_group::1 (the scan's form).  1: CTA pairs, cta_group::2 with M = 256, each CTA holding
+ *                  half of the second operand (an even number of CTAs is launched).
+ *   iters          1 .. 2^24.
+ *   status_device  DEVICE, one int the caller zeroed; LT_STATUS_TIMEOUT is OR-ed in if a bounded wait ran out.
+ * Only enqueues on `stream`; returns LT_ERR_INVALID_ARG for bad arguments, LT_ERR_CUDA if the launch fails.
+ */
+int lt_debug_umma_stream(int pair, int iters, int* status_device, void* stream);
+
+/*
  * Instrumentation (no counterpart in the paper; used by the benchmark).
  *   lt_launch_count     kernels this library has launched so far in this process.
  *   lt_set_profiling    when enabled, lt_indexer_topk(_ex) on the fused path records CUDA events on

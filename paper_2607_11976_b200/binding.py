@@ -109,6 +109,8 @@ def load() -> ctypes.CDLL:
     lib.lt_read_status_static.restype = i
     lib.lt_debug_wait_timeout.argtypes = [i, ip, vp]
     lib.lt_debug_wait_timeout.restype = i
+    lib.lt_debug_umma_stream.argtypes = [i, i, ip, vp]
+    lib.lt_debug_umma_stream.restype = i
     lib.lt_indexer_topk_strided.argtypes = [i, vp, fp, vp, ctypes.c_longlong, fp, i, i, i, i, i, i, ip, fp, vp, sz,
                                             ctypes.POINTER(Tunables), vp]
     lib.lt_indexer_topk_strided.restype = i
@@ -325,6 +327,11 @@ def lt_read_status_static(stream=None) -> list:
 def lt_debug_wait_timeout(limit_us: int, result2, stream=None) -> None:
     """Runs the bounded-wait probe: result2 (int32 CUDA tensor of 2) receives (wait result, abort flag)."""
     _check(load().lt_debug_wait_timeout(int(limit_us), _ptr(result2), _stream(stream)), "lt_debug_wait_timeout")
+
+
+def lt_debug_umma_stream(pair: bool, iters: int, status, stream=None) -> None:
+    """Enqueues one launch of the bare FP8 UMMA stream; status: zeroed int32 CUDA tensor of 1."""
+    _check(load().lt_debug_umma_stream(1 if pair else 0, int(iters), _ptr(status), _stream(stream)), "lt_debug_umma_stream")
 
 
 def lt_launch_count() -> int:

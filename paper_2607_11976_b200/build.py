@@ -10,7 +10,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB_DIR = os.path.join(HERE, "lib")
 LIB_PATH = os.path.join(LIB_DIR, "liblt_indexer.so")
 DEBUG_LIB_PATH = os.path.join(LIB_DIR, "liblt_indexer_dbg.so")  # bounds-checking build (-DLT_DEBUG_BOUNDS)
-SOURCES = ["lt_api.cu", "lt_scan_mma.cu", "lt_scan_fp8.cu", "lt_select.cu", "lt_sampler.cu", "lt_dsa_union.cu", "lt_scan_knn.cu"]
+SOURCES = ["lt_api.cu", "lt_scan_mma.cu", "lt_scan_fp8.cu", "lt_select.cu", "lt_sampler.cu", "lt_dsa_union.cu", "lt_scan_knn.cu", "lt_umma_stream.cu"]
 HEADERS = ["lt_common.cuh", "lt_host.h", "lt_ptx.cuh", os.path.join("..", "..", "include", "lt_indexer.h")]
 
 

@@ -1027,6 +1027,15 @@ int lt_debug_wait_timeout(int limit_us, int* result2_device, void* stream) {
   return LT_OK;
 }
 
+int lt_debug_umma_stream(int pair, int iters, int* status_device, void* stream) {
+  if (iters <= 0 || iters > (1 << 24) || status_device == nullptr) return LT_ERR_INVALID_ARG;
+  int grid = sm_count();
+  if (pair) grid &= ~1;
+  if (grid <= 0) return LT_ERR_CUDA;
+  LT_LAUNCH(launch_umma_stream(pair != 0, iters, status_device, grid, static_cast<cudaStream_t>(stream)));
+  return LT_OK;
+}
+
 unsigned long long lt_launch_count(void) { return g_launches.load(); }
 
 int lt_set_profiling(int enable) {

@@ -72,6 +72,8 @@ cudaError_t launch_scan_fp8(int mode, const void* q, int T, const void* k, long 
 // One warp waits, with the bounded wait every scan kernel uses, on a barrier nobody arrives at:
 // result2[0] = what the wait returned (0 = gave up), result2[1] = the abort flag it left behind.
 cudaError_t launch_wait_timeout_probe(unsigned int limit_us, int* result2, cudaStream_t stream);
+// bare FP8 UMMA stream (measurement aid): grid CTAs, an even number when pair is set
+cudaError_t launch_umma_stream(bool pair, int iters, int* status, int grid, cudaStream_t stream);
 
 // q: [T][64][128]; k: view of n_keys_view rows whose pitch is key_pitch_elems elements.
 cudaError_t launch_scan_mma(int dtype, int mode, const void* q, int T, const void* k, long long n_keys_view,
