@@ -779,7 +779,7 @@ cudaError_t launch_sample_stats(const float* sample, int T, int n_sample, int ra
 cudaError_t launch_final_select(const FinalSelectParams& p, cudaStream_t stream) {
   // room for every candidate at or above the final threshold edge: k plus the population of the threshold bin,
   // which for a small k over millions of keys can be several thousand (the select that follows cuts them to k)
-  int sel_cap = next_pow2(4 * p.topk);
+  int sel_cap = next_pow2(2 * p.topk);
   if (sel_cap < 8192) sel_cap = 8192;
   if (sel_cap > kSelCap) sel_cap = kSelCap;
   const int smem = sel_cap * static_cast<int>(sizeof(uint64_t));
