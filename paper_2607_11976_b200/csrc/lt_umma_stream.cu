@@ -3,8 +3,9 @@
 // stay in shared memory - no TMA, no epilogue, the accumulators are never read.  What this stream sustains is the
 // ceiling of the tensor roofline the scan kernels are held against on the same board, at the clocks and the power the
 // board grants it.  Two forms: one CTA per SM (cta_group::1, M 128 x N 256, the scan's form) and CTA pairs
-// (cta_group::2, M 256 x N 256: each CTA holds its own 128 rows of A and half of B, the leader issues, the commit is
-// multicast to both CTAs' barriers).  Both do 2 x 128 x 256 x 128 x 2 flops per SM and iteration.
+// (cta_group::2, M 256 x N 256: each CTA holds its own 128 rows of A and half of B; the leader issues, follows the
+// completions on its own barriers, and the peer waits for it at the closing cluster barrier).  Both do
+// 2 x 128 x 256 x 128 x 2 flops per SM and iteration.
 #include "lt_host.h"
 #include "lt_ptx.cuh"
 
@@ -41,12 +42,9 @@ __device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, ui
       "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// the barrier at the same shared-memory offset in every CTA of the mask gets one arrival when the UMMAs issued so far
-// have completed
-__device__ __forceinline__ void tc_commit_pair(uint32_t bar, uint16_t cta_mask) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
-               "h"(cta_mask)
-               : "memory");
+// one arrival on the issuing CTA's barrier when the pair's UMMAs issued so far have completed
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
 template <bool kPair>
@@ -98,12 +96,12 @@ __global__ void __launch_bounds__(kStreamThreads, 1) umma_stream_kernel(int iter
     // instruction descriptor: fp32 accumulators, e4m3 x e4m3, N = 256, M = 128 (256 over the pair)
     constexpr uint32_t idesc = (1u << 4) | (static_cast<uint32_t>(256 >> 3) << 17) | (static_cast<uint32_t>((kPair ? 256 : 128) >> 4) << 24);
     bool ok = true;
-    // two iterations in flight: iteration it waits for the commit of iteration it - 2 on the same barrier.  Both
-    // CTAs of a pair follow the phases (the commit reaches both), only the leader issues.
-    for (int it = 0; it < iters + 2 && ok; ++it) {
-      if (it >= 2) ok = mbar_wait<20>(smem_u32(&st->bar[it & 1]), ((it - 2) >> 1) & 1, abort_flag);
-      if (!ok || it >= iters) continue;
-      if (!kPair || rank == 0) {
+    // two iterations in flight: iteration it waits for the commit of iteration it - 2 on the same barrier.  Of a
+    // pair only the leader issues and waits; its peer goes straight to the closing cluster barrier.
+    if (!kPair || rank == 0) {
+      for (int it = 0; it < iters + 2 && ok; ++it) {
+        if (it >= 2) ok = mbar_wait<20>(smem_u32(&st->bar[it & 1]), ((it - 2) >> 1) & 1, abort_flag);
+        if (!ok || it >= iters) continue;
         tc_fence_after();
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
@@ -115,7 +113,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) umma_stream_kernel(int iter
             else tc_mma<true>(tmem_base + u * 256, a, b, idesc, kb > 0 ? 1u : 0u);
           }
         }
-        if (kPair) tc_commit_pair(smem_u32(&st->bar[it & 1]), 3);
+        if (kPair) tc_commit_pair(smem_u32(&st->bar[it & 1]));
         else tc_commit(smem_u32(&st->bar[it & 1]));
       }
     }
