@@ -237,7 +237,10 @@ int pick_seg_tiles(const Tun& tun, int n_keys, int n_blocks, int grid) {
   if (tun.segment_tiles > 0) return tun.segment_tiles;
   int n_tiles = (n_keys + kTileKeys - 1) / kTileKeys;
   int seg = 256;
-  while (seg > 16 && static_cast<long long>(n_blocks) * ((n_tiles + seg - 1) / seg) < 2ll * grid) seg >>= 1;
+  // at least two items per CTA, so that rows of different visible length even out; one per CTA for a chunk of one
+  // or two row blocks, whose items all have the same length (measured: 84 instead of 102 us for 1 row over 2^20 keys)
+  const long long want = (n_blocks <= 2 ? 1ll : 2ll) * grid;
+  while (seg > 16 && static_cast<long long>(n_blocks) * ((n_tiles + seg - 1) / seg) < want) seg >>= 1;
   // Work items are dealt to the persistent CTAs round-robin, so the launch lasts as long as the CTA with the
   // most items: among the sizes from the one above down to 16 tiles, take the shortest such critical path (in key
   // tiles, plus a few tiles' worth of per-item start-up: the query block of an item is as large as four key tiles).
