@@ -232,7 +232,9 @@ __device__ __forceinline__ void flush_stage(const uint2* list, int count, const 
   __syncwarp();
 }
 
-template <bool kFp8, int kMode, bool kPaged>
+// kU: units in use.  A chunk of at most kUnitQ rows (a decode step, a tail of a few tokens) has no row for the second
+// unit: its launch issues, loads and finishes unit 0 only, which halves the tensor and the epilogue work per key tile.
+template <bool kFp8, int kMode, bool kPaged, int kU = kUnits>
 __global__ void __launch_bounds__(kThreads, 1)
 scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k, const ScanParams p) {
   using C = Cfg<kFp8>;
@@ -304,8 +306,8 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         // query block: wait until the UMMAs of the previous item no longer read it
         ok = mbar_wait<40>(smem_u32(&st->bar_q_empty), (n_done & 1) ^ 1, abort_flag);
         if (!ok) break;
-        mbar_arrive_expect_tx(smem_u32(&st->bar_q_full), C::kQBytes);
-        for (int u = 0; u < kUnits; ++u)
+        mbar_arrive_expect_tx(smem_u32(&st->bar_q_full), kU * C::kHalves * kQTile);
+        for (int u = 0; u < kU; ++u)
           for (int hf = 0; hf < C::kHalves; ++hf)
             tma_load_2d(q_base + (u * C::kHalves + hf) * kQTile, &tm_q, hf * C::kElemsPerRow128,
                         (it.t0 + u * kUnitQ) * kH, smem_u32(&st->bar_q_full));
@@ -361,7 +363,7 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         for (int tile = it.tile_lo; tile < it.tile_hi && ok; ++tile) {
           ok = mbar_wait<40>(smem_u32(&st->bar_full[stage]), phase, abort_flag);
           if (!ok) break;
-          for (int u = 0; u < kUnits; ++u) {
+          for (int u = 0; u < kU; ++u) {
             ok = mbar_wait<40>(smem_u32(&st->bar_tmem_empty[u]), acc_phase ^ 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
@@ -521,7 +523,7 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           // keys of this tile that some row of the block may not see (diagonal or ragged last tile)
           const bool partial = (tile + 1) * kTileKeys > vis_first;
 #pragma unroll
-          for (int u = 0; u < kUnits; ++u) {
+          for (int u = 0; u < kU; ++u) {
             const int r = u * kUnitQ + g;
             float thr = 0.f;
             if (kMode == kModeFilter) thr = *reinterpret_cast<volatile float*>(&st->thr[r]);
@@ -576,7 +578,7 @@ scan_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         }
         if (kMode == kModeFilter) {
 #pragma unroll
-          for (int u = 0; u < kUnits; ++u)
+          for (int u = 0; u < kU; ++u)
             if (cnt[u] > 0) {
               const int r = u * kUnitQ + g;
               flush_stage(st->stage[ew][u], cnt[u], p, it.t0 + r, lane, st->smin[r], st->width[r], st->inv_width[r]);
@@ -639,19 +641,24 @@ bool make_map(CUtensorMap* map, bool fp8, const void* base, uint64_t rows, uint6
   return r == CUDA_SUCCESS;
 }
 
-template <bool kFp8, int kMode, bool kPaged>
+template <bool kFp8, int kMode, bool kPaged, int kU>
 cudaError_t launch_one(const CUtensorMap& tq, const CUtensorMap& tk, const ScanParams& p, int grid, cudaStream_t stream) {
   constexpr int bytes = smem_bytes<kFp8>();
-  cudaError_t e = cudaFuncSetAttribute(scan_kernel<kFp8, kMode, kPaged>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  cudaError_t e = cudaFuncSetAttribute(scan_kernel<kFp8, kMode, kPaged, kU>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
   if (e != cudaSuccess) return e;
-  scan_kernel<kFp8, kMode, kPaged><<<grid, kThreads, bytes, stream>>>(tq, tk, p);
+  scan_kernel<kFp8, kMode, kPaged, kU><<<grid, kThreads, bytes, stream>>>(tq, tk, p);
   return cudaGetLastError();
 }
-// the paged variant is a separate instantiation so that the dense kernels carry none of its address arithmetic
+// the paged variant is a separate instantiation so that the dense kernels carry none of its address arithmetic; the
+// one-unit variant exists for the fused scan of a chunk of at most kUnitQ rows
 template <bool kFp8, int kMode>
 cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const ScanParams& p, int grid, cudaStream_t stream) {
-  return p.page_table != nullptr ? launch_one<kFp8, kMode, true>(tq, tk, p, grid, stream)
-                                 : launch_one<kFp8, kMode, false>(tq, tk, p, grid, stream);
+  if (kMode == kModeFilter && p.fb_list == nullptr && p.row_end - p.row_begin <= kUnitQ) {
+    return p.page_table != nullptr ? launch_one<kFp8, kModeFilter, true, 1>(tq, tk, p, grid, stream)
+                                   : launch_one<kFp8, kModeFilter, false, 1>(tq, tk, p, grid, stream);
+  }
+  return p.page_table != nullptr ? launch_one<kFp8, kMode, true, kUnits>(tq, tk, p, grid, stream)
+                                 : launch_one<kFp8, kMode, false, kUnits>(tq, tk, p, grid, stream);
 }
 
 }  // namespace

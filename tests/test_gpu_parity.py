@@ -281,6 +281,23 @@ def test_random_shapes_fused_path():
         assert_own_scores_rule(inp, idx, score, dumped, range(T))
 
 
+@pytest.mark.parametrize("name", ["dsa_bf16", "fp8_ar1"])
+@pytest.mark.parametrize("T", [1, 2, 4, 5])
+def test_chunks_of_a_few_rows(name, T):
+    """Decode-like chunks.  Up to four rows take the one-unit launch of the fused scan (only the first accumulator half
+    is issued and finished), five rows the regular one; the dump that arbitrates always runs the regular kernel, so the
+    own-scores rule also shows that both launches produce the same score bits."""
+    inp = make_config(name, T=T, N=50000, topk=777)
+    idx, score, status = run_topk(inp, lt.Tunables(path=lt.LT_PATH_FUSED))
+    assert status[0] & lt.LT_STATUS_TIMEOUT == 0
+    dumped = dump_scores(inp, 0, T, lt.LT_PATH_FUSED)
+    assert_matches_oracle(inp, idx, score, list(range(T)), dumped, 0)
+    # a forced overflow sends the rows through the exact fallback: same bits
+    idx2, score2, status2 = run_topk(inp, lt.Tunables(path=lt.LT_PATH_FUSED, cap_mult=1, sample_rank=1))
+    assert status2[1] > 0
+    assert np.array_equal(idx2, idx) and np.array_equal(score2.view(np.uint32), score.view(np.uint32))
+
+
 def test_soak_random_problems_with_random_tunables():
     """A wider seeded sweep than the test above: eight recipes, chunks of 1 - 400 rows, up to 600,000 keys, any causal
     offset, k up to 4096, random capacity / sample size / sample rank / work-item length / grid.  The arbiter is the
